@@ -1,0 +1,119 @@
+/* fp8attn -- FP8 in-context-learning (ICL) attention for tabular foundation
+ * models on NVIDIA B200 (sm_100a).  C ABI of libfp8attn.so.
+ *
+ * Conventions shared by every entry point
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; the library
+ *     allocates no device memory and keeps no pointer after a call returns.
+ *   - Tensors are dense row-major [B, H, rows, d] with d innermost; base
+ *     addresses must be 16-byte aligned.  bf16 tensors hold IEEE bfloat16 bit
+ *     patterns, FP8 tensors hold e4m3fn codes (1-4-3, bias 7, no infinities,
+ *     0x7F/0xFF = NaN, largest finite value 448).
+ *   - `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).  All
+ *     work is enqueued on it; no entry point synchronises the host unless its
+ *     description says so.
+ *   - `workspace` is caller-owned device memory of at least
+ *     fp8attn_workspace_bytes(...) bytes, 256-byte aligned, that must have been
+ *     zero-filled once before its first use (cudaMemset).  Calls that share a
+ *     workspace must be ordered on one stream; overlapping them races.
+ *   - Return value: an fp8attn_status_t.  Argument errors are detected on the
+ *     host before anything is launched.  Device-side problems (a bounded wait
+ *     that ran out) are recorded in the workspace and read back with
+ *     fp8attn_last_device_status(); the kernels never trap or spin forever.
+ *   - Supported head dims: d = 64 and d = 128.  n_train >= 1, n_test >= 0.
+ */
+#ifndef FP8ATTN_H_
+#define FP8ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FP8ATTN_OK = 0,
+    FP8ATTN_ERR_INVALID_ARG = 1, /* null pointer, bad size, misaligned address   */
+    FP8ATTN_ERR_UNSUPPORTED = 2, /* head dim other than 64/128, device not sm_100 */
+    FP8ATTN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small    */
+    FP8ATTN_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed           */
+    FP8ATTN_ERR_TIMEOUT = 5      /* a device-side bounded wait expired            */
+} fp8attn_status_t;
+
+/* Per-head absmax quantization to e4m3 (paper Eq. 2, Method section).
+ *
+ *   s[b,h]  = max_{r,c} |x[b,h,r,c]| / 448        (fp32, IEEE division; 1.0 for an all-zero head)
+ *   x8      = round_to_nearest_even_e4m3( clamp( x / s, -448, 448 ) )   (fp32 IEEE division)
+ *
+ *   x_bf16   in   bf16 [B,H,rows,d]
+ *   scale_in in   NULL            -> the scale is computed from x itself (train queries, keys, values)
+ *                 fp32 [B,H]      -> this scale is used instead and values outside its range saturate at
+ *                                    +-448: the paper's shared train-query scale for the test queries,
+ *                                    which keeps test predictions independent of the test batch.
+ *   x_fp8    out  e4m3 [B,H,rows,d]
+ *   scale_out out fp32 [B,H], the dequantization scale actually used (may be NULL when scale_in is given)
+ *
+ * rows may be 0 (nothing is written except scale_out when scale_in is given).
+ * Inputs containing NaN or infinity are not supported.
+ */
+int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d,
+                     const float* scale_in, void* x_fp8, float* scale_out,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Fused FP8 ICL attention (paper Eq. 1 with the Method section's two-call
+ * structure and quantization placement).
+ *
+ * For every (b,h): the n_train train queries attend to all n_train train keys
+ * (non-causal, the diagonal included) and the n_test test queries attend to the
+ * same n_train train keys only; both read the same quantized K and V.
+ *
+ *   S   = Q8 K8^T                         FP8 tensor-core product, fp32 accumulation
+ *   x   = softmax_scale * s_q * s_k * S   (the Q and K scales are folded into the softmax scale)
+ *   P   = exp(x - rowmax) lifted by 2^8 and rounded to e4m3 inside the kernel
+ *         (the row maximum maps to 256 < 448); the normaliser sums the unrounded fp32 values
+ *   out = bf16( s_v * (P8 V8) / rowsum )  (the V scale is applied in the epilogue)
+ *
+ *   q_train_fp8 in  e4m3 [B,H,n_train,d]     q_test_fp8 in e4m3 [B,H,n_test,d] (NULL iff n_test == 0)
+ *   k_fp8,v_fp8 in  e4m3 [B,H,n_train,d]
+ *   scale_q/k/v in  fp32 [B,H] device arrays (scale_q serves train AND test queries)
+ *   softmax_scale   <= 0 selects 1/sqrt(d)
+ *   out_train_bf16 out bf16 [B,H,n_train,d]  out_test_bf16 out bf16 [B,H,n_test,d] (NULL iff n_test == 0)
+ */
+int fp8attn_icl_forward(const void* q_train_fp8, const void* q_test_fp8,
+                        const void* k_fp8, const void* v_fp8,
+                        const float* scale_q, const float* scale_k, const float* scale_v,
+                        int B, int H, int64_t n_train, int64_t n_test, int d,
+                        float softmax_scale,
+                        void* out_train_bf16, void* out_test_bf16,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The same ICL attention on unquantized bf16 Q/K/V with bf16 probabilities: the
+ * 16-bit comparison path (the paper's "ours 16-bit" control in its latency
+ * tables).  Arguments as above without scales; all tensors bf16.
+ */
+int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k, const void* v,
+                         int B, int H, int64_t n_train, int64_t n_test, int d,
+                         float softmax_scale,
+                         void* out_train_bf16, void* out_test_bf16,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of workspace the three calls above need for these sizes (a few KB). */
+size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t n_test, int d);
+
+/* Synchronises `cuda_stream`, reads and clears the device status word of
+ * `workspace`, and returns it (FP8ATTN_OK, FP8ATTN_ERR_TIMEOUT, or
+ * FP8ATTN_ERR_CUDA if the stream reported an error).  `detail`, if not NULL,
+ * receives a kernel-specific code saying which wait expired.  For tests. */
+int fp8attn_last_device_status(void* workspace, void* cuda_stream, uint32_t* detail);
+
+/* Static, human-readable name of a status code. */
+const char* fp8attn_status_string(int status);
+
+/* Number of kernels the library has launched in this process so far (all
+ * entry points, all threads).  Used by benchmarks to report launch counts. */
+uint64_t fp8attn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP8ATTN_H_ */

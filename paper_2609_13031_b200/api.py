@@ -1,0 +1,178 @@
+"""Python binding of libfp8attn.so (declared in ``include/fp8attn.h``).
+
+Argument marshalling only: every function hands device pointers, sizes and the
+current CUDA stream to the C-ABI entry point of the same name.  torch is used
+for device memory and streams.  There is no fallback: if the CUDA library has
+not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfp8attn.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+
+EXPORTS = (
+    "fp8attn_quantize", "fp8attn_icl_forward", "bf16attn_icl_forward",
+    "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
+    "fp8attn_launch_count",
+)
+
+_lib = None
+
+
+class Fp8AttnError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status_string(status)} (status {status})")
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it is missing (build it with
+    ``python -m paper_2609_13031_b200.build`` or ``__graft_entry__.build()``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} not found: the CUDA extension has not been built and there is no "
+            "CPU fallback.  Run `python -m paper_2609_13031_b200.build`.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float,
+                             ctypes.c_size_t)
+    lib.fp8attn_quantize.restype = i32
+    lib.fp8attn_quantize.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp, sz, vp]
+    lib.fp8attn_icl_forward.restype = i32
+    lib.fp8attn_icl_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i64, i32, f32,
+                                        vp, vp, vp, sz, vp]
+    lib.bf16attn_icl_forward.restype = i32
+    lib.bf16attn_icl_forward.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, vp, vp, vp,
+                                         sz, vp]
+    lib.fp8attn_workspace_bytes.restype = sz
+    lib.fp8attn_workspace_bytes.argtypes = [i32, i32, i64, i64, i32]
+    lib.fp8attn_last_device_status.restype = i32
+    lib.fp8attn_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.fp8attn_status_string.restype = ctypes.c_char_p
+    lib.fp8attn_status_string.argtypes = [i32]
+    lib.fp8attn_launch_count.restype = ctypes.c_uint64
+    lib.fp8attn_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().fp8attn_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(load().fp8attn_launch_count())
+
+
+def _ptr(t: torch.Tensor | None):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(fn: str, rc: int):
+    if rc != OK:
+        raise Fp8AttnError(fn, rc)
+
+
+def workspace_bytes(B: int, H: int, n_train: int = 0, n_test: int = 0, d: int = 64) -> int:
+    return int(load().fp8attn_workspace_bytes(B, H, n_train, n_test, d))
+
+
+def new_workspace(B: int, H: int, device="cuda") -> torch.Tensor:
+    """A zero-filled workspace tensor for tensors with B*H heads."""
+    return torch.zeros(workspace_bytes(B, H), dtype=torch.uint8, device=device)
+
+
+def _dims(x: torch.Tensor):
+    assert x.dim() == 4 and x.is_cuda and x.is_contiguous(), "expected contiguous CUDA [B,H,rows,d]"
+    return x.shape
+
+
+def quantize(x: torch.Tensor, workspace: torch.Tensor, scale_in: torch.Tensor | None = None,
+             out: torch.Tensor | None = None, scale_out: torch.Tensor | None = None):
+    """fp8attn_quantize: bf16 [B,H,rows,d] -> (e4m3 codes as uint8 [B,H,rows,d], fp32 scale [B,H])."""
+    B, H, rows, d = _dims(x)
+    assert x.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty((B, H, rows, d), dtype=torch.uint8, device=x.device)
+    if scale_out is None:
+        scale_out = torch.empty((B, H), dtype=torch.float32, device=x.device)
+    if scale_in is not None:
+        assert scale_in.dtype == torch.float32 and scale_in.is_contiguous() and scale_in.numel() == B * H
+    rc = load().fp8attn_quantize(_ptr(x), B, H, rows, d, _ptr(scale_in), _ptr(out), _ptr(scale_out),
+                                 _ptr(workspace), workspace.numel(), _stream())
+    _check("fp8attn_quantize", rc)
+    return out, scale_out
+
+
+def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
+                    softmax_scale: float = 0.0, out_train=None, out_test=None):
+    """fp8attn_icl_forward on uint8 e4m3 tensors; returns (out_train, out_test) bf16."""
+    B, H, n_train, d = _dims(k)
+    n_test = 0 if q_test is None else q_test.shape[2]
+    for t in (q_train, k, v):
+        assert t.dtype == torch.uint8
+    if out_train is None:
+        out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
+    if out_test is None and n_test > 0:
+        out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+    rc = load().fp8attn_icl_forward(
+        _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v),
+        _ptr(scale_q), _ptr(scale_k), _ptr(scale_v), B, H, n_train, n_test, d,
+        float(softmax_scale), _ptr(out_train), _ptr(out_test) if n_test else None,
+        _ptr(workspace), workspace.numel(), _stream())
+    _check("fp8attn_icl_forward", rc)
+    return out_train, out_test
+
+
+def icl_forward_bf16(q_train, q_test, k, v, workspace, softmax_scale: float = 0.0,
+                     out_train=None, out_test=None):
+    """bf16attn_icl_forward on bf16 tensors; returns (out_train, out_test) bf16."""
+    B, H, n_train, d = _dims(k)
+    n_test = 0 if q_test is None else q_test.shape[2]
+    for t in (q_train, k, v):
+        assert t.dtype == torch.bfloat16
+    if out_train is None:
+        out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
+    if out_test is None and n_test > 0:
+        out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+    rc = load().bf16attn_icl_forward(
+        _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v), B, H, n_train, n_test, d,
+        float(softmax_scale), _ptr(out_train), _ptr(out_test) if n_test else None,
+        _ptr(workspace), workspace.numel(), _stream())
+    _check("bf16attn_icl_forward", rc)
+    return out_train, out_test
+
+
+def last_device_status(workspace: torch.Tensor):
+    """Synchronise the current stream; returns (status, detail) recorded by the kernels."""
+    detail = ctypes.c_uint32(0)
+    rc = load().fp8attn_last_device_status(_ptr(workspace), _stream(), ctypes.byref(detail))
+    return int(rc), int(detail.value)
+
+
+def icl_attention(q_train, q_test, k, v, workspace=None, softmax_scale: float = 0.0):
+    """The whole hot path on bf16 inputs: quantize Q_train, K, V per head, quantize
+    Q_test with the train-query scale, then the fused FP8 attention."""
+    B, H, _, _ = _dims(k)
+    if workspace is None:
+        workspace = new_workspace(B, H, k.device)
+    q8, sq = quantize(q_train, workspace)
+    k8, sk = quantize(k, workspace)
+    v8, sv = quantize(v, workspace)
+    t8 = None
+    if q_test is not None and q_test.shape[2] > 0:
+        t8, _ = quantize(q_test, workspace, scale_in=sq)
+    return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale)

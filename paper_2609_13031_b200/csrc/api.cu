@@ -1,0 +1,140 @@
+// extern "C" entry points of libfp8attn.so: argument checking and dispatch.
+#include <atomic>
+#include <math.h>
+
+#include "common.h"
+
+namespace fp8attn {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_shape(int B, int H, int d) {
+    if (B <= 0 || H <= 0) return FP8ATTN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return FP8ATTN_ERR_UNSUPPORTED;
+    return FP8ATTN_OK;
+}
+
+int check_workspace(const void* ws, size_t bytes, int B, int H) {
+    if (ws == nullptr || !aligned(ws, 256) || bytes < workspace_bytes(B, H)) return FP8ATTN_ERR_WORKSPACE;
+    return FP8ATTN_OK;
+}
+
+// The kernels are built for sm_100a only.
+int check_device() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return FP8ATTN_ERR_CUDA;
+    return major == 10 ? FP8ATTN_OK : FP8ATTN_ERR_UNSUPPORTED;
+}
+
+int forward(bool fp8, const void* q_train, const void* q_test, const void* k, const void* v,
+            const float* sq, const float* sk, const float* sv, int B, int H, int64_t n_train,
+            int64_t n_test, int d, float softmax_scale, void* out_train, void* out_test,
+            void* workspace, size_t workspace_bytes_, void* stream) {
+    int rc = check_shape(B, H, d);
+    if (rc != FP8ATTN_OK) return rc;
+    if (n_train < 1 || n_test < 0 || n_train > 0x7fffff00ll || n_test > 0x7fffff00ll)
+        return FP8ATTN_ERR_INVALID_ARG;
+    if (!q_train || !k || !v || !out_train) return FP8ATTN_ERR_INVALID_ARG;
+    if (n_test > 0 && (!q_test || !out_test)) return FP8ATTN_ERR_INVALID_ARG;
+    if (fp8 && (!sq || !sk || !sv)) return FP8ATTN_ERR_INVALID_ARG;
+    if (!aligned(q_train, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out_train, 16) ||
+        (n_test > 0 && (!aligned(q_test, 16) || !aligned(out_test, 16))))
+        return FP8ATTN_ERR_INVALID_ARG;
+    if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return FP8ATTN_ERR_INVALID_ARG;
+    rc = check_workspace(workspace, workspace_bytes_, B, H);
+    if (rc != FP8ATTN_OK) return rc;
+    rc = check_device();
+    if (rc != FP8ATTN_OK) return rc;
+    AttnParams p;
+    p.q_train = q_train; p.q_test = q_test; p.k = k; p.v = v;
+    p.scale_q = sq; p.scale_k = sk; p.scale_v = sv;
+    p.B = B; p.H = H; p.n_train = n_train; p.n_test = n_test; p.d = d;
+    p.softmax_scale = softmax_scale;
+    p.out_train = out_train; p.out_test = out_test;
+    p.status = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsStatusOffset);
+    return launch_icl_attention(p, fp8, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+}  // namespace fp8attn
+
+using namespace fp8attn;
+
+extern "C" {
+
+int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d, const float* scale_in,
+                     void* x_fp8, float* scale_out, void* workspace, size_t workspace_bytes_,
+                     void* cuda_stream) {
+    int rc = check_shape(B, H, d);
+    if (rc != FP8ATTN_OK) return rc;
+    if (rows < 0) return FP8ATTN_ERR_INVALID_ARG;
+    if (rows > 0 && (!x_bf16 || !x_fp8)) return FP8ATTN_ERR_INVALID_ARG;
+    if (!scale_in && !scale_out) return FP8ATTN_ERR_INVALID_ARG;
+    if (!aligned(x_bf16, 16) || !aligned(x_fp8, 16) || !aligned(scale_in, 4) || !aligned(scale_out, 4))
+        return FP8ATTN_ERR_INVALID_ARG;
+    rc = check_workspace(workspace, workspace_bytes_, B, H);
+    if (rc != FP8ATTN_OK) return rc;
+    rc = check_device();
+    if (rc != FP8ATTN_OK) return rc;
+    uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
+    return launch_quantize(x_bf16, (int64_t)B * H, rows * (int64_t)d, scale_in, x_fp8, scale_out, amax,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
+int fp8attn_icl_forward(const void* q_train_fp8, const void* q_test_fp8, const void* k_fp8,
+                        const void* v_fp8, const float* scale_q, const float* scale_k,
+                        const float* scale_v, int B, int H, int64_t n_train, int64_t n_test, int d,
+                        float softmax_scale, void* out_train_bf16, void* out_test_bf16,
+                        void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    return forward(true, q_train_fp8, q_test_fp8, k_fp8, v_fp8, scale_q, scale_k, scale_v, B, H, n_train,
+                   n_test, d, softmax_scale, out_train_bf16, out_test_bf16, workspace, workspace_bytes_,
+                   cuda_stream);
+}
+
+int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k, const void* v, int B,
+                         int H, int64_t n_train, int64_t n_test, int d, float softmax_scale,
+                         void* out_train_bf16, void* out_test_bf16, void* workspace,
+                         size_t workspace_bytes_, void* cuda_stream) {
+    return forward(false, q_train, q_test, k, v, nullptr, nullptr, nullptr, B, H, n_train, n_test, d,
+                   softmax_scale, out_train_bf16, out_test_bf16, workspace, workspace_bytes_, cuda_stream);
+}
+
+size_t fp8attn_workspace_bytes(int B, int H, int64_t, int64_t, int) {
+    if (B <= 0 || H <= 0) return 0;
+    return workspace_bytes(B, H);
+}
+
+int fp8attn_last_device_status(void* workspace, void* cuda_stream, uint32_t* detail) {
+    if (!workspace) return FP8ATTN_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    uint32_t words[2] = {0, 0};
+    if (cudaMemcpy(words, workspace, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return FP8ATTN_ERR_CUDA;
+    if (detail) *detail = words[1];
+    if (words[0] != 0 && cudaMemset(workspace, 0, sizeof(words)) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    return (int)words[0];
+}
+
+const char* fp8attn_status_string(int status) {
+    switch (status) {
+        case FP8ATTN_OK: return "ok";
+        case FP8ATTN_ERR_INVALID_ARG: return "invalid argument";
+        case FP8ATTN_ERR_UNSUPPORTED: return "unsupported head dimension, size or device";
+        case FP8ATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case FP8ATTN_ERR_CUDA: return "CUDA call failed";
+        case FP8ATTN_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+uint64_t fp8attn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

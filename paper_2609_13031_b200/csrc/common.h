@@ -1,0 +1,43 @@
+// Internal declarations shared by the translation units of libfp8attn.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "fp8attn.h"
+
+namespace fp8attn {
+
+// Workspace layout (device memory, caller-owned, zero-filled once):
+//   [0,4)    device status word (fp8attn_status_t, 0 = ok); first error wins
+//   [4,8)    detail code of that error (which wait expired, which CTA)
+//   [256, 256 + 4*B*H)  per-(b,h) absmax accumulators (fp32 bit patterns) of the
+//                       quantizer; cleared at the start of every quantize call
+constexpr size_t kWsStatusOffset = 0;
+constexpr size_t kWsDetailOffset = 4;
+constexpr size_t kWsAmaxOffset = 256;
+
+inline size_t workspace_bytes(int B, int H) {
+    size_t amax = (size_t)4 * (size_t)B * (size_t)H;
+    return kWsAmaxOffset + ((amax + 255) / 256) * 256;
+}
+
+void count_launch();
+
+// quantize.cu
+int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
+                    const float* scale_in, void* x_fp8, float* scale_out,
+                    uint32_t* amax_bits, cudaStream_t stream);
+
+// attention.cu
+struct AttnParams {
+    const void* q_train; const void* q_test; const void* k; const void* v;
+    const float* scale_q; const float* scale_k; const float* scale_v;  // NULL for bf16
+    int B, H; int64_t n_train, n_test; int d;
+    float softmax_scale;
+    void* out_train; void* out_test;
+    uint32_t* status;  // workspace status words
+};
+int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream);
+
+}  // namespace fp8attn

@@ -1,0 +1,151 @@
+// Per-head absmax quantization of bf16 tensors to e4m3 (paper Eq. 2).
+//
+// Two HBM-bound kernels per call:
+//   absmax_kernel    max |x| per head, packed bf16x2 max, one atomicMax per block
+//   quantize_kernel  s = amax/448, y = x/s (IEEE fp32), cvt.rn.satfinite.e4m3x2
+// Algorithmic traffic: 2 B read per element for the maximum, 2 B read + 1 B
+// written for the conversion (5 B per element; 3 B when the scale is given).
+// The conversion walks each head backwards so that it starts on the part of the
+// head the maximum pass touched last, which is still in L2.
+#include <cuda_bf16.h>
+
+#include "common.h"
+
+namespace fp8attn {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) {
+    return *reinterpret_cast<__nv_bfloat162*>(&u);
+}
+
+// grid: (blocks_per_head, n_heads).  A head is vecs_per_head 16-byte vectors.
+__global__ void __launch_bounds__(kThreads)
+absmax_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, uint32_t* __restrict__ amax_bits) {
+    const uint4* xh = x + (int64_t)blockIdx.y * vecs_per_head;
+    __nv_bfloat162 m = as_bf162(0u);
+    int64_t stride = (int64_t)gridDim.x * kThreads;
+    int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    for (; i + 3 * stride < vecs_per_head; i += 4 * stride) {
+        uint4 a = ld_nc_v4(xh + i), b = ld_nc_v4(xh + i + stride);
+        uint4 c = ld_nc_v4(xh + i + 2 * stride), e = ld_nc_v4(xh + i + 3 * stride);
+        __nv_bfloat162 m0 = __hmax2(__habs2(as_bf162(a.x)), __habs2(as_bf162(a.y)));
+        __nv_bfloat162 m1 = __hmax2(__habs2(as_bf162(a.z)), __habs2(as_bf162(a.w)));
+        __nv_bfloat162 m2 = __hmax2(__habs2(as_bf162(b.x)), __habs2(as_bf162(b.y)));
+        __nv_bfloat162 m3 = __hmax2(__habs2(as_bf162(b.z)), __habs2(as_bf162(b.w)));
+        __nv_bfloat162 m4 = __hmax2(__habs2(as_bf162(c.x)), __habs2(as_bf162(c.y)));
+        __nv_bfloat162 m5 = __hmax2(__habs2(as_bf162(c.z)), __habs2(as_bf162(c.w)));
+        __nv_bfloat162 m6 = __hmax2(__habs2(as_bf162(e.x)), __habs2(as_bf162(e.y)));
+        __nv_bfloat162 m7 = __hmax2(__habs2(as_bf162(e.z)), __habs2(as_bf162(e.w)));
+        m = __hmax2(m, __hmax2(__hmax2(__hmax2(m0, m1), __hmax2(m2, m3)),
+                               __hmax2(__hmax2(m4, m5), __hmax2(m6, m7))));
+    }
+    for (; i < vecs_per_head; i += stride) {
+        uint4 a = ld_nc_v4(xh + i);
+        m = __hmax2(m, __hmax2(__hmax2(__habs2(as_bf162(a.x)), __habs2(as_bf162(a.y))),
+                               __hmax2(__habs2(as_bf162(a.z)), __habs2(as_bf162(a.w)))));
+    }
+    // |x| as a non-negative fp32 bit pattern orders like an unsigned integer
+    float f = fmaxf(__low2float(m), __high2float(m));
+    uint32_t bits = __float_as_uint(f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bits = max(bits, __shfl_xor_sync(0xffffffffu, bits, o));
+    __shared__ uint32_t warp_max[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bits;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        bits = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) bits = max(bits, __shfl_xor_sync(0xffffffffu, bits, o));
+        if (threadIdx.x == 0) atomicMax(amax_bits + blockIdx.y, bits);
+    }
+}
+
+// two floats -> two e4m3 codes (lo in bits 0..7, hi in bits 8..15), RNE, saturating
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return (uint32_t)r;
+}
+
+__device__ __forceinline__ uint32_t quant4(uint32_t w0, uint32_t w1, float s) {
+    // w0, w1: four bf16 values; an fp32 with the bf16 bits in its upper half is that value
+    float a = __fdiv_rn(__uint_as_float(w0 << 16), s);
+    float b = __fdiv_rn(__uint_as_float(w0 & 0xffff0000u), s);
+    float c = __fdiv_rn(__uint_as_float(w1 << 16), s);
+    float e = __fdiv_rn(__uint_as_float(w1 & 0xffff0000u), s);
+    return cvt_e4m3x2(a, b) | (cvt_e4m3x2(c, e) << 16);
+}
+
+// grid: (blocks_per_head, n_heads).  Each thread turns 32 B of bf16 into 16 B of
+// e4m3 per step.  pairs_per_head = elems_per_head / 16.
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const uint4* __restrict__ x, int64_t pairs_per_head,
+                const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
+                uint4* __restrict__ out, float* __restrict__ scale_out) {
+    float s;
+    if (scale_in != nullptr) {
+        s = scale_in[blockIdx.y];
+    } else {
+        float amax = __uint_as_float(amax_bits[blockIdx.y]);
+        s = amax == 0.0f ? 1.0f : __fdiv_rn(amax, 448.0f);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0 && scale_out != nullptr) scale_out[blockIdx.y] = s;
+    const uint4* xh = x + (int64_t)blockIdx.y * pairs_per_head * 2;
+    uint4* oh = out + (int64_t)blockIdx.y * pairs_per_head;
+    int64_t stride = (int64_t)gridDim.x * kThreads;
+    // walk the head from its end towards its start
+    for (int64_t r = (int64_t)blockIdx.x * kThreads + threadIdx.x; r < pairs_per_head; r += stride) {
+        int64_t i = pairs_per_head - 1 - r;
+        uint4 a = ld_nc_v4(xh + 2 * i), b = ld_nc_v4(xh + 2 * i + 1);
+        uint4 o;
+        o.x = quant4(a.x, a.y, s);
+        o.y = quant4(a.z, a.w, s);
+        o.z = quant4(b.x, b.y, s);
+        o.w = quant4(b.z, b.w, s);
+        oh[i] = o;
+    }
+}
+
+}  // namespace
+
+int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
+                    const float* scale_in, void* x_fp8, float* scale_out,
+                    uint32_t* amax_bits, cudaStream_t stream) {
+    if (n_heads <= 0) return FP8ATTN_OK;
+    if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
+    const int64_t vecs = elems_per_head / 8, pairs = elems_per_head / 16;
+    // enough blocks to fill 148 SMs several times over, never more than the work
+    auto blocks_for = [&](int64_t units) {
+        int64_t want = (148 * 16 + n_heads - 1) / n_heads;
+        int64_t have = (units + kThreads - 1) / kThreads;
+        int64_t b = want < have ? want : have;
+        return (unsigned)(b < 1 ? 1 : b);
+    };
+    if (scale_in == nullptr) {
+        if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * n_heads, stream) != cudaSuccess)
+            return FP8ATTN_ERR_CUDA;
+        if (elems_per_head > 0) {
+            absmax_kernel<<<dim3(blocks_for((vecs + 3) / 4), (unsigned)n_heads), kThreads, 0, stream>>>(
+                (const uint4*)x_bf16, vecs, amax_bits);
+            count_launch();
+        }
+    }
+    // also launched for empty heads when the scale must be written out
+    if (elems_per_head > 0 || scale_out != nullptr) {
+        quantize_kernel<<<dim3(blocks_for(pairs), (unsigned)n_heads), kThreads, 0, stream>>>(
+            (const uint4*)x_bf16, pairs, scale_in, amax_bits, (uint4*)x_fp8, scale_out);
+        count_launch();
+    }
+    return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
+}
+
+}  // namespace fp8attn

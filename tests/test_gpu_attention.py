@@ -1,0 +1,181 @@
+"""GPU parity: fused ICL attention (FP8 and BF16 paths) against the oracle's exact
+softmax attention over the dequantized / original operands."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (bf16_bits_to_f64, check_bf16_attention, check_fp8_attention,
+                     f32_to_bf16_bits, sample_rows)
+from paper_2609_13031_b200 import api
+from paper_2609_13031_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def out_to_f64(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def oracle_quantized(g):
+    q8, sq = oracle.quantize(g["q_train"])
+    k8, sk = oracle.quantize(g["k"])
+    v8, sv = oracle.quantize(g["v"])
+    t8 = None
+    if g["q_test"].shape[2]:
+        t8, _ = oracle.quantize(g["q_test"], scale_in=sq)
+    return dict(q8=q8, k8=k8, v8=v8, t8=t8, sq=sq, sk=sk, sv=sv)
+
+
+def gpu_fp8_forward(z, w, alpha=0.0):
+    dev = lambda a: None if a is None else torch.from_numpy(a).cuda()
+    ws = api.new_workspace(w.B, w.H)
+    o_tr, o_te = api.icl_forward_fp8(dev(z["q8"]), dev(z["t8"]), dev(z["k8"]), dev(z["v8"]),
+                                     dev(z["sq"]), dev(z["sk"]), dev(z["sv"]), ws, alpha)
+    assert api.last_device_status(ws) == (0, 0)
+    return o_tr, o_te
+
+
+def check_fp8_case(w, n_sample=None, diffuse=False, alpha=None):
+    g = W.generate(w)
+    z = oracle_quantized(g)
+    o_tr, o_te = gpu_fp8_forward(z, w, 0.0 if alpha is None else alpha)
+    stats = {}
+    for name, out, q8, nq in (("train", o_tr, z["q8"], w.n_train), ("test", o_te, z["t8"], w.n_test)):
+        if nq == 0:
+            assert out is None
+            continue
+        rows = np.arange(nq) if n_sample is None else sample_rows(nq, n_sample, w.seed)
+        A, Abs, Bnd = oracle.icl_attention_rows(q8, z["k8"], z["v8"], rows, sq=z["sq"], sk=z["sk"],
+                                                sv=z["sv"], alpha=alpha)
+        got = out_to_f64(out[:, :, torch.from_numpy(rows).cuda()])
+        stats[name] = check_fp8_attention(got, A, Abs, Bnd, diffuse, label=f"{w.name}/{name}")
+        # no worse than the method-faithful two-pass e4m3-P evaluation
+        O4 = oracle.icl_attention_rows(q8, z["k8"], z["v8"], rows, sq=z["sq"], sk=z["sk"],
+                                       sv=z["sv"], alpha=alpha, mode="p8")
+        faithful = np.mean(np.abs(O4 - A) / np.maximum(1, Abs))
+        assert stats[name]["mean_norm"] <= 1.25 * faithful + 1e-5, (stats[name], faithful)
+    return stats
+
+
+def check_bf16_case(w, n_sample=None):
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    q_test = to_dev(g["q_test"]) if w.n_test else None
+    o_tr, o_te = api.icl_forward_bf16(to_dev(g["q_train"]), q_test, to_dev(g["k"]), to_dev(g["v"]), ws)
+    assert api.last_device_status(ws) == (0, 0)
+    for name, out, q, nq in (("train", o_tr, g["q_train"], w.n_train), ("test", o_te, g["q_test"], w.n_test)):
+        if nq == 0:
+            continue
+        rows = np.arange(nq) if n_sample is None else sample_rows(nq, n_sample, w.seed)
+        A, Abs, _ = oracle.icl_attention_rows(q, g["k"], g["v"], rows)
+        got = out_to_f64(out[:, :, torch.from_numpy(rows).cuda()])
+        check_bf16_attention(got, A, Abs, label=f"{w.name}/{name}")
+
+
+# ---- FP8 path ---------------------------------------------------------------------
+
+def test_fp8_c1_full():
+    check_fp8_case(W.CONFIGS["C1"], diffuse=True)
+
+
+@pytest.mark.parametrize("n,m", [(1, 0), (1, 1), (5, 3), (127, 1), (128, 128), (129, 77), (255, 257),
+                                 (500, 77), (640, 0), (1000, 300)])
+def test_fp8_ragged_shapes(n, m):
+    check_fp8_case(W.CONFIGS["C1"].scaled(n, m))
+
+
+def test_fp8_d128_small():
+    check_fp8_case(W.CONFIGS["C3"].scaled(700, 130))
+
+
+def test_fp8_c2_sampled():
+    check_fp8_case(W.CONFIGS["C2"], n_sample=96)
+
+
+def test_fp8_c4_like_shifted_keys_diffuse():
+    check_fp8_case(W.CONFIGS["C4"].scaled(2048, 300), n_sample=64, diffuse=True)
+
+
+def test_fp8_c3_full_size_sampled():
+    check_fp8_case(W.CONFIGS["C3"], n_sample=40)
+
+
+def test_fp8_custom_softmax_scale():
+    check_fp8_case(W.CONFIGS["C1"].scaled(300, 40), alpha=0.05)
+
+
+# ---- BF16 comparison path -----------------------------------------------------------
+
+def test_bf16_c1_full():
+    check_bf16_case(W.CONFIGS["C1"])
+
+
+@pytest.mark.parametrize("n,m", [(1, 0), (129, 77), (500, 300)])
+def test_bf16_ragged_shapes(n, m):
+    check_bf16_case(W.CONFIGS["C1"].scaled(n, m))
+
+
+def test_bf16_d128_small():
+    check_bf16_case(W.CONFIGS["C3"].scaled(700, 130))
+
+
+def test_bf16_c2_sampled():
+    check_bf16_case(W.CONFIGS["C2"], n_sample=64)
+
+
+# ---- structure of the ICL layer -------------------------------------------------------
+
+def test_test_rows_are_batch_invariant_and_share_kv_with_train_rows():
+    w = W.CONFIGS["C1"].scaled(384, 200)
+    g = W.generate(w)
+    z = oracle_quantized(g)
+    _, full = gpu_fp8_forward(z, w)
+    # a single test row alone gives the bit-identical output row
+    z1 = dict(z); z1["t8"] = np.ascontiguousarray(z["t8"][:, :, 131:132])
+    _, single = gpu_fp8_forward(z1, w.scaled(384, 1))
+    assert torch.equal(single[:, :, 0], full[:, :, 131])
+    # permuting the test batch permutes the outputs and nothing else
+    perm = np.random.default_rng(0).permutation(w.n_test)
+    z2 = dict(z); z2["t8"] = np.ascontiguousarray(z["t8"][:, :, perm])
+    tr2, shuffled = gpu_fp8_forward(z2, w)
+    assert torch.equal(shuffled, full[:, :, torch.from_numpy(perm).cuda()])
+    # a test query identical to a train query produces the train row's output
+    z3 = dict(z); t8 = z["t8"].copy(); t8[:, :, 5] = z["q8"][:, :, 300]; z3["t8"] = t8
+    tr3, te3 = gpu_fp8_forward(z3, w)
+    assert torch.equal(te3[:, :, 5], tr3[:, :, 300])
+    # train outputs never depend on the test queries
+    assert torch.equal(tr2, tr3)
+
+
+def test_runs_are_deterministic():
+    w = W.CONFIGS["C2"].scaled(1024, 256)
+    z = oracle_quantized(W.generate(w))
+    a = gpu_fp8_forward(z, w)
+    b = gpu_fp8_forward(z, w)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_forward_argument_errors():
+    lib = api.load()
+    ws = api.new_workspace(1, 1)
+    q = torch.zeros((1, 1, 8, 64), dtype=torch.uint8, device="cuda")
+    o = torch.zeros((1, 1, 8, 64), dtype=torch.bfloat16, device="cuda")
+    s = torch.ones((1, 1), dtype=torch.float32, device="cuda")
+    p = lambda t: t.data_ptr()
+    f = lib.fp8attn_icl_forward
+    args = lambda **kw: [kw.get("q", p(q)), None, p(q), p(q), p(s), p(s), kw.get("sv", p(s)), 1, 1,
+                         kw.get("n", 8), kw.get("m", 0), kw.get("d", 64), 0.0, p(o), None, p(ws),
+                         kw.get("wsb", ws.numel()), None]
+    assert f(*args(d=32)) == api.ERR_UNSUPPORTED
+    assert f(*args(n=0)) == api.ERR_INVALID_ARG
+    assert f(*args(m=4)) == api.ERR_INVALID_ARG          # test rows without test tensors
+    assert f(*args(sv=None)) == api.ERR_INVALID_ARG
+    assert f(*args(q=None)) == api.ERR_INVALID_ARG
+    assert f(*args(wsb=16)) == api.ERR_WORKSPACE
+    assert f(*args()) == api.OK
+    assert api.last_device_status(ws) == (0, 0)

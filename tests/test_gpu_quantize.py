@@ -1,0 +1,111 @@
+"""GPU parity: fp8attn_quantize must match the oracle bit for bit (codes and scales)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import f32_to_bf16_bits
+from paper_2609_13031_b200 import api
+from paper_2609_13031_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def run_case(w):
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    scales = {}
+    for name in ("q_train", "k", "v"):
+        codes, s = api.quantize(to_dev(g[name]), ws)
+        rc, rs = oracle.quantize(g[name])
+        assert np.array_equal(s.cpu().numpy(), rs), name
+        got = codes.cpu().numpy()
+        assert np.array_equal(got, rc), (name, int((got != rc).sum()))
+        scales[name] = s
+    if w.n_test:
+        codes, s = api.quantize(to_dev(g["q_test"]), ws, scale_in=scales["q_train"])
+        rc, rs = oracle.quantize(g["q_test"], scale_in=scales["q_train"].cpu().numpy())
+        assert np.array_equal(s.cpu().numpy(), rs)
+        assert np.array_equal(codes.cpu().numpy(), rc)
+    assert api.last_device_status(ws) == (0, 0)
+
+
+@pytest.mark.parametrize("cfg", ["C1", "C2"])
+def test_full_configs_small(cfg):
+    run_case(W.CONFIGS[cfg])
+
+
+@pytest.mark.parametrize("cfg,n,m", [("C3", 8192, 2048), ("C4", 4096, 1000), ("C5", 16384, 4096),
+                                      ("C1", 1, 0), ("C1", 3, 1), ("C2", 129, 77), ("C3", 500, 7)])
+def test_scaled_and_ragged(cfg, n, m):
+    run_case(W.CONFIGS[cfg].scaled(n, m))
+
+
+@pytest.mark.parametrize("cfg", ["C3", "C4", "C5"])
+def test_full_size(cfg):
+    """Full-size tensors, one tensor at a time to bound host memory."""
+    w = W.CONFIGS[cfg]
+    ws = api.new_workspace(w.B, w.H)
+    sq = None
+    for name, tid, rows in (("q_train", W.Q_TRAIN, w.n_train), ("k", W.K, w.n_train),
+                            ("v", W.V, w.n_train), ("q_test", W.Q_TEST, w.n_test)):
+        bits = W.fill(np.empty((w.B, w.H, rows, w.d), dtype=np.uint16), w, tid)
+        s_in = sq if name == "q_test" else None
+        codes, s = api.quantize(to_dev(bits), ws, scale_in=s_in)
+        rc, rs = oracle.quantize(bits, scale_in=None if s_in is None else s_in.cpu().numpy())
+        if name == "q_train":
+            sq = s
+        assert np.array_equal(s.cpu().numpy(), rs), name
+        got = codes.cpu().numpy()
+        assert np.array_equal(got, rc), (name, int((got != rc).sum()))
+        del bits, codes, got, rc
+    assert api.last_device_status(ws) == (0, 0)
+
+
+def test_special_values_and_edges():
+    ws = api.new_workspace(1, 3)
+    x = np.zeros((1, 3, 16, 64), dtype=np.float32)
+    x[0, 1] = np.linspace(-3, 3, 1024, dtype=np.float32).reshape(16, 64)
+    x[0, 2, :, :] = 1e-30                      # tiny magnitudes: scale is subnormal-adjacent
+    x[0, 2, 3, 5] = -3e-30
+    x[0, 1, 0, 0] = -0.0
+    bits = f32_to_bf16_bits(x)
+    codes, s = api.quantize(to_dev(bits), ws)
+    rc, rs = oracle.quantize(bits)
+    assert np.array_equal(s.cpu().numpy(), rs) and np.array_equal(codes.cpu().numpy(), rc)
+    assert rs[0, 0] == 1.0
+    # test queries beyond the train range saturate at +-448
+    big = f32_to_bf16_bits(np.full((1, 3, 2, 64), 1e6, dtype=np.float32))
+    big[0, :, 1] |= 0x8000
+    codes, s2 = api.quantize(to_dev(big), ws, scale_in=s)
+    rc, _ = oracle.quantize(big, scale_in=rs)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert set(np.unique(rc[0, 1])) == {0x7E, 0xFE}
+    # heads are independent: scaling one head leaves the others' codes untouched
+    y = x.copy(); y[0, 1] *= 1024
+    c2, s3 = api.quantize(to_dev(f32_to_bf16_bits(y)), ws)
+    c1, _ = api.quantize(to_dev(bits), ws)
+    assert torch.equal(c1[0, 0], c2[0, 0]) and torch.equal(c1[0, 2], c2[0, 2]) and torch.equal(c1[0, 1], c2[0, 1])
+
+
+def test_argument_errors_are_reported_on_the_host():
+    lib = api.load()
+    ws = api.new_workspace(1, 2)
+    x = torch.zeros((1, 2, 4, 64), dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros((1, 2, 4, 64), dtype=torch.uint8, device="cuda")
+    s = torch.zeros((1, 2), dtype=torch.float32, device="cuda")
+    p = lambda t: t.data_ptr()
+    q = lib.fp8attn_quantize
+    assert q(p(x), 1, 2, 4, 96, None, p(o), p(s), p(ws), ws.numel(), None) == api.ERR_UNSUPPORTED
+    assert q(None, 1, 2, 4, 64, None, p(o), p(s), p(ws), ws.numel(), None) == api.ERR_INVALID_ARG
+    assert q(p(x), 0, 2, 4, 64, None, p(o), p(s), p(ws), ws.numel(), None) == api.ERR_INVALID_ARG
+    assert q(p(x), 1, 2, 4, 64, None, p(o), None, p(ws), ws.numel(), None) == api.ERR_INVALID_ARG
+    assert q(p(x) + 2, 1, 2, 4, 64, None, p(o), p(s), p(ws), ws.numel(), None) == api.ERR_INVALID_ARG
+    assert q(p(x), 1, 2, 4, 64, None, p(o), p(s), p(ws), 8, None) == api.ERR_WORKSPACE
+    assert q(p(x), 1, 2, 4, 64, None, p(o), p(s), None, ws.numel(), None) == api.ERR_WORKSPACE
+    assert q(p(x), 1, 2, 4, 64, None, p(o), p(s), p(ws), ws.numel(), None) == api.OK
+    torch.cuda.synchronize()
