@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 ICL-attention hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+quantize Q_train, K, V (per-head absmax), quantize Q_test with the train-query
+scale, then the fused train->train + test->train FP8 attention.  The metric is
+tensor-core TFLOPS, 4*B*H*d*N*(N+M) FLOPs per step divided by the step time
+(quantization included, as in the paper's latency tables).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no
+exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+NOMINAL_FP8_OVER_BF16 = 2.0           # dense tensor peak ratio (4.5 / 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.stop_flag = threading.Event()
+        self.sm, self.max_sm, self.reasons = [], 0.0, set()
+
+    def sample(self):
+        try:
+            out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                 timeout=5).stdout.strip().splitlines()[0]
+            f = [x.strip() for x in out.split(",")]
+            self.sm.append(float(f[0]))
+            self.max_sm = float(f[1])
+            for name, val in zip(self.NAMES, f[2:]):
+                if val.lower().startswith("active"):
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self.stop_flag.is_set():
+            self.sample()
+            self.stop_flag.wait(0.2)
+
+    def result(self):
+        self.stop_flag.set()
+        self.join(timeout=10)
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_sm,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def oracle_sample(w, rows_per_head: int, seed: int = 0):
+    """Time the CPU oracle, as it stands, on a bounded sample of workload ``w``:
+    the full per-head quantization of K, V and both query tensors, then exact
+    attention for ``rows_per_head`` train and test query rows per (b,h) against
+    all train keys.  Returns (TFLOPS of the sampled attention rows, info)."""
+    import oracle
+    from paper_2609_13031_b200 import workloads as W
+    oracle.build()
+    g = W.generate(w)
+    cores = oracle.hardware_threads()
+    t0 = time.perf_counter()
+    q8, sq = oracle.quantize(g["q_train"])
+    k8, sk = oracle.quantize(g["k"])
+    v8, sv = oracle.quantize(g["v"])
+    t8, _ = oracle.quantize(g["q_test"], scale_in=sq)
+    t_quant = time.perf_counter() - t0
+    rng = np.random.default_rng(seed)
+    n_rows = 0
+    t0 = time.perf_counter()
+    for q, nq in ((q8, w.n_train), (t8, w.n_test)):
+        if nq == 0:
+            continue
+        rows = np.unique(rng.integers(0, nq, size=min(rows_per_head, nq)))
+        oracle.icl_attention_rows(q, k8, v8, rows, sq=sq, sk=sk, sv=sv)
+        n_rows += rows.size * w.B * w.H
+    t_attn = time.perf_counter() - t0
+    flops = 4.0 * w.d * w.n_train * n_rows
+    # quantization is charged in proportion to the sampled share of the query rows
+    share = n_rows / float(w.B * w.H * (w.n_train + w.n_test))
+    seconds = t_attn + t_quant * share
+    info = {"cores": cores, "rows": int(n_rows), "seconds_attention": t_attn,
+            "seconds_quantize_full": t_quant,
+            "sample": f"{n_rows} query rows ({rows_per_head} train + {rows_per_head} test per head) "
+                      f"against all {w.n_train} train keys of {w.name}, plus the sampled share of a "
+                      f"full quantization pass"}
+    return flops / seconds / 1e12, info
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle, timed on the host cores, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals, info = [], None
+    for i in range(args.warmup + args.steps):
+        v, info = oracle_sample(w, args.ref_rows, seed=i)
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    sec = info["seconds_attention"]
+    print(json.dumps({
+        "impl": "reference", "metric": "fp8_icl_attention_tflops", "value": value, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * sec, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "n_train": w.n_train,
+                   "n_test": w.n_test},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
+                         "sample": info["sample"]},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=96, help="oracle sample: query rows per head and call")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-bf16", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2609_13031_b200 import workloads as W
+    w = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_13031_b200 import api
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    api.load()                      # raises if the CUDA library is missing: no fallback
+    peaks, peak_kind = load_peaks()
+
+    # ---- inputs: seeded synthetic bf16 tensors, generated on the host into pinned memory ----
+    host = {}
+    for name, tid, rows in (("q_train", W.Q_TRAIN, w.n_train), ("k", W.K, w.n_train),
+                            ("v", W.V, w.n_train), ("q_test", W.Q_TEST, w.n_test)):
+        t = torch.empty((w.B, w.H, rows, w.d), dtype=torch.int16).pin_memory()
+        W.fill(t.numpy().view(np.uint16), w, tid)
+        host[name] = t.view(torch.bfloat16)
+    dev = {k: torch.empty_like(v, device="cuda") for k, v in host.items()}
+    for k in host:
+        dev[k].copy_(host[k], non_blocking=True)
+    ws = api.new_workspace(w.B, w.H)
+    shape_tr, shape_te = (w.B, w.H, w.n_train, w.d), (w.B, w.H, w.n_test, w.d)
+    buf = {
+        "q8": torch.empty(shape_tr, dtype=torch.uint8, device="cuda"),
+        "k8": torch.empty(shape_tr, dtype=torch.uint8, device="cuda"),
+        "v8": torch.empty(shape_tr, dtype=torch.uint8, device="cuda"),
+        "t8": torch.empty(shape_te, dtype=torch.uint8, device="cuda"),
+        "sq": torch.empty((w.B, w.H), dtype=torch.float32, device="cuda"),
+        "sk": torch.empty((w.B, w.H), dtype=torch.float32, device="cuda"),
+        "sv": torch.empty((w.B, w.H), dtype=torch.float32, device="cuda"),
+        "st": torch.empty((w.B, w.H), dtype=torch.float32, device="cuda"),
+        "o_tr": torch.empty(shape_tr, dtype=torch.bfloat16, device="cuda"),
+        "o_te": torch.empty(shape_te, dtype=torch.bfloat16, device="cuda"),
+    }
+    host_out = {"o_tr": torch.empty(shape_tr, dtype=torch.bfloat16).pin_memory(),
+                "o_te": torch.empty(shape_te, dtype=torch.bfloat16).pin_memory()}
+
+    def quantize_all():
+        api.quantize(dev["q_train"], ws, out=buf["q8"], scale_out=buf["sq"])
+        api.quantize(dev["k"], ws, out=buf["k8"], scale_out=buf["sk"])
+        api.quantize(dev["v"], ws, out=buf["v8"], scale_out=buf["sv"])
+        api.quantize(dev["q_test"], ws, scale_in=buf["sq"], out=buf["t8"], scale_out=buf["st"])
+
+    def attention_fp8():
+        api.icl_forward_fp8(buf["q8"], buf["t8"], buf["k8"], buf["v8"], buf["sq"], buf["sk"], buf["sv"],
+                            ws, 0.0, out_train=buf["o_tr"], out_test=buf["o_te"])
+
+    def attention_bf16():
+        api.icl_forward_bf16(dev["q_train"], dev["q_test"], dev["k"], dev["v"], ws, 0.0,
+                             out_train=buf["o_tr"], out_test=buf["o_te"])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing: K steps, events per sub-kernel group ----
+    for _ in range(args.warmup):
+        quantize_all()
+        attention_fp8()
+    sync_all()
+    status = api.last_device_status(ws)
+    if status != (0, 0):
+        raise RuntimeError(f"device status {status}")
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = api.launch_count()
+    marks = []
+    sync_all()
+    e_start, e_end = ev(), ev()
+    e_start.record()
+    for _ in range(args.steps):
+        a, b, c = ev(), ev(), ev()
+        a.record()
+        quantize_all()
+        b.record()
+        attention_fp8()
+        c.record()
+        marks.append((a, b, c))
+    e_end.record()
+    sync_all()
+    launches = api.launch_count() - launches0
+    clocks = sampler.result()
+    total_ms = max_over_ranks(e_start.elapsed_time(e_end))
+    ms_step = total_ms / args.steps
+    ms_quant = float(np.mean([a.elapsed_time(b) for a, b, _ in marks]))
+    ms_attn = float(np.mean([b.elapsed_time(c) for _, b, c in marks]))
+    status = api.last_device_status(ws)
+    if status != (0, 0):
+        raise RuntimeError(f"device status {status}")
+
+    # ---- the in-build BF16 path on the same inputs ----
+    ms_bf16 = None
+    if not args.no_bf16:
+        for _ in range(2):
+            attention_bf16()
+        sync_all()
+        a, b = ev(), ev()
+        n_bf = max(2, min(args.steps, 5))
+        a.record()
+        for _ in range(n_bf):
+            attention_bf16()
+        b.record()
+        sync_all()
+        ms_bf16 = max_over_ranks(a.elapsed_time(b)) / n_bf
+
+    # ---- end to end: pinned host inputs -> device -> path -> host outputs, every step ----
+    def e2e_step():
+        for k in host:
+            dev[k].copy_(host[k], non_blocking=True)
+        quantize_all()
+        attention_fp8()
+        host_out["o_tr"].copy_(buf["o_tr"], non_blocking=True)
+        host_out["o_te"].copy_(buf["o_te"], non_blocking=True)
+
+    e2e_step()
+    sync_all()
+    n_e2e = max(2, min(args.steps, 5))
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    b.record()
+    sync_all()
+    ms_e2e = max_over_ranks(a.elapsed_time(b)) / n_e2e
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, info = oracle_sample(w, args.ref_rows)
+        cpu_baseline = {"value": v, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
+                        "sample": info["sample"]}
+
+    if rank == 0:
+        flops = w.flops
+        tf_step = world * flops / (ms_step * 1e-3) / 1e12
+        tf_attn = flops / (ms_attn * 1e-3) / 1e12
+        peak_fp8 = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops_sustained"]
+        peak_fp8_burst = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops"]
+        quant_bytes = w.B * w.H * w.d * (5 * 3 * w.n_train + 3 * w.n_test)
+        line = {
+            "metric": "fp8_icl_attention_tflops", "value": tf_step, "unit": "TFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: B={w.B} H={w.H} d={w.d} n_train={w.n_train} n_test={w.n_test}",
+                       "step": "quantize Q_train,K,V,Q_test + fused FP8 ICL attention",
+                       "l2": "inputs larger than L2 (bf16 inputs %.0f MB)" % (h2d / 1e6),
+                       "replicas": world},
+            "clocks": clocks,
+            "e2e": {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "kernel": "icl_attention_kernel<fp8>",
+                         "achieved": tf_attn, "peak": peak_fp8, "unit": "TFLOP/s",
+                         "frac": tf_attn / peak_fp8, "traffic": None,
+                         "peak_source": f"2 x bf16_tflops_sustained ({peak_kind}), nominal fp8:bf16 ratio",
+                         "frac_of_burst_peak": tf_attn / peak_fp8_burst,
+                         "frac_of_nominal_4500": tf_attn / 4500.0},
+            "cpu_baseline": cpu_baseline,
+            "breakdown": {
+                "ms_quantize": ms_quant, "ms_attention_fp8": ms_attn, "ms_attention_bf16": ms_bf16,
+                "attention_fp8_tflops": tf_attn,
+                "attention_bf16_tflops": None if ms_bf16 is None else flops / (ms_bf16 * 1e-3) / 1e12,
+                "speedup_vs_bf16_attention_only": None if ms_bf16 is None else ms_bf16 / ms_attn,
+                "speedup_vs_bf16_with_quantize": None if ms_bf16 is None else ms_bf16 / (ms_attn + ms_quant),
+                "quantize_gbs": quant_bytes / (ms_quant * 1e-3) / 1e9,
+                "quantize_frac_of_hbm": quant_bytes / (ms_quant * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "paper_context": "up to 1.72x (d=64) / 1.82x (d=128) FP8 over 16-bit kernels on RTX PRO 6000",
+            },
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
