@@ -40,7 +40,7 @@ def gpu_fp8_forward(z, w, alpha=0.0):
     return o_tr, o_te
 
 
-def check_fp8_case(w, n_sample=None, diffuse=False, alpha=None):
+def check_fp8_case(w, n_sample=None, diffuse=False, alpha=None, named_config=False):
     g = W.generate(w)
     z = oracle_quantized(g)
     o_tr, o_te = gpu_fp8_forward(z, w, 0.0 if alpha is None else alpha)
@@ -53,7 +53,8 @@ def check_fp8_case(w, n_sample=None, diffuse=False, alpha=None):
         A, Abs, Bnd = oracle.icl_attention_rows(q8, z["k8"], z["v8"], rows, sq=z["sq"], sk=z["sk"],
                                                 sv=z["sv"], alpha=alpha)
         got = out_to_f64(out[:, :, torch.from_numpy(rows).cuda()])
-        stats[name] = check_fp8_attention(got, A, Abs, Bnd, diffuse, label=f"{w.name}/{name}")
+        stats[name] = check_fp8_attention(got, A, Abs, Bnd, diffuse, label=f"{w.name}/{name}",
+                                          named_config=named_config)
         # no worse than the method-faithful two-pass e4m3-P evaluation
         O4 = oracle.icl_attention_rows(q8, z["k8"], z["v8"], rows, sq=z["sq"], sk=z["sk"],
                                        sv=z["sv"], alpha=alpha, mode="p8")
@@ -80,7 +81,7 @@ def check_bf16_case(w, n_sample=None):
 # ---- FP8 path ---------------------------------------------------------------------
 
 def test_fp8_c1_full():
-    check_fp8_case(W.CONFIGS["C1"], diffuse=True)
+    check_fp8_case(W.CONFIGS["C1"], diffuse=True, named_config=True)
 
 
 @pytest.mark.parametrize("n,m", [(1, 0), (1, 1), (5, 3), (127, 1), (128, 128), (129, 77), (255, 257),
@@ -94,7 +95,7 @@ def test_fp8_d128_small():
 
 
 def test_fp8_c2_sampled():
-    check_fp8_case(W.CONFIGS["C2"], n_sample=96)
+    check_fp8_case(W.CONFIGS["C2"], n_sample=96, named_config=True)
 
 
 def test_fp8_c4_like_shifted_keys_diffuse():
@@ -102,7 +103,7 @@ def test_fp8_c4_like_shifted_keys_diffuse():
 
 
 def test_fp8_c3_full_size_sampled():
-    check_fp8_case(W.CONFIGS["C3"], n_sample=40)
+    check_fp8_case(W.CONFIGS["C3"], n_sample=40, named_config=True)
 
 
 def test_fp8_custom_softmax_scale():
