@@ -37,7 +37,9 @@ typedef enum {
     FP8ATTN_ERR_UNSUPPORTED = 2, /* head dim other than 64/128, device not sm_100 */
     FP8ATTN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small    */
     FP8ATTN_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed           */
-    FP8ATTN_ERR_TIMEOUT = 5      /* a device-side bounded wait expired            */
+    FP8ATTN_ERR_TIMEOUT = 5,     /* a device-side bounded wait expired            */
+    FP8ATTN_ERR_TOO_LARGE = 6    /* more heads than the built-in scratch of the
+                                    allocation-free entry point can hold          */
 } fp8attn_status_t;
 
 /* Per-head absmax quantization to e4m3 (paper Eq. 2, Method section).
@@ -96,6 +98,37 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
                          float softmax_scale,
                          void* out_train_bf16, void* out_test_bf16,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Allocation-free quantizer (the paper has no counterpart; this is a
+ * packaging variant of fp8attn_quantize, same arithmetic, same results).
+ *
+ * Some hosts can give this library nothing but input and output buffers and may
+ * not allocate device memory on its behalf: an inference runtime's plugin slot
+ * that has no workspace argument, a serving process whose memory pool already
+ * owns all of HBM (a cudaMalloc there fails or fragments the pool), or a
+ * latency-critical loop that cannot afford the device-wide synchronisation
+ * cudaMalloc implies.  For them the per-head absmax accumulators live in a
+ * fixed array inside the library image instead of a caller-provided workspace.
+ * The array holds FP8ATTN_NOALLOC_MAX_HEADS 32-bit slots (16 KiB) and stays
+ * resident on every GPU that loads the library until the process exits.
+ *
+ *   - Arguments as fp8attn_quantize, without the workspace.  The caller still
+ *     passes x_bf16, x_fp8 and scale_out (device pointers it owns).
+ *   - B*H > FP8ATTN_NOALLOC_MAX_HEADS returns FP8ATTN_ERR_TOO_LARGE and
+ *     launches nothing.
+ *   - The call performs no cudaMalloc / cudaFree and calls no allocating
+ *     library routine.  The first call on each device looks up the device
+ *     address of the built-in array (cudaGetSymbolAddress, with that device
+ *     current); make that first call outside any stream capture.
+ *   - Every call on a device shares the one array and the array keeps the last
+ *     call's contents: each call clears the slots it uses before accumulating,
+ *     and two calls that overlap on the GPU (different streams, no ordering
+ *     between them) race on it.  Order them on one stream or with events.
+ */
+#define FP8ATTN_NOALLOC_MAX_HEADS 4096
+int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int d,
+                             const float* scale_in, void* x_fp8, float* scale_out,
+                             void* cuda_stream);
 
 /* Bytes of workspace the three calls above need for these sizes (a few KB). */
 size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t n_test, int d);

@@ -15,12 +15,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfp8attn.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = range(7)
+NOALLOC_MAX_HEADS = 4096
 
 EXPORTS = (
     "fp8attn_quantize", "fp8attn_icl_forward", "bf16attn_icl_forward",
     "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
-    "fp8attn_launch_count",
+    "fp8attn_launch_count", "fp8attn_quantize_noalloc",
 )
 
 _lib = None
@@ -47,6 +48,8 @@ def load() -> ctypes.CDLL:
                              ctypes.c_size_t)
     lib.fp8attn_quantize.restype = i32
     lib.fp8attn_quantize.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp, sz, vp]
+    lib.fp8attn_quantize_noalloc.restype = i32
+    lib.fp8attn_quantize_noalloc.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp]
     lib.fp8attn_icl_forward.restype = i32
     lib.fp8attn_icl_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i64, i32, f32,
                                         vp, vp, vp, sz, vp]
@@ -114,6 +117,22 @@ def quantize(x: torch.Tensor, workspace: torch.Tensor, scale_in: torch.Tensor | 
     rc = load().fp8attn_quantize(_ptr(x), B, H, rows, d, _ptr(scale_in), _ptr(out), _ptr(scale_out),
                                  _ptr(workspace), workspace.numel(), _stream())
     _check("fp8attn_quantize", rc)
+    return out, scale_out
+
+
+def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor,
+                     scale_in: torch.Tensor | None = None):
+    """fp8attn_quantize_noalloc: like ``quantize`` but with no workspace; the
+    scratch it needs is built into the library.  For hosts that may not allocate
+    device memory, the caller passes every buffer (``out``: uint8 like ``x``,
+    ``scale_out``: fp32 [B,H]) and this wrapper allocates nothing either.  At
+    most ``NOALLOC_MAX_HEADS`` heads; calls on one device must not overlap."""
+    B, H, rows, d = _dims(x)
+    assert x.dtype == torch.bfloat16 and out.dtype == torch.uint8 and out.shape == x.shape
+    assert scale_out.dtype == torch.float32 and scale_out.numel() == B * H
+    rc = load().fp8attn_quantize_noalloc(_ptr(x), B, H, rows, d, _ptr(scale_in), _ptr(out),
+                                         _ptr(scale_out), _stream())
+    _check("fp8attn_quantize_noalloc", rc)
     return out, scale_out
 
 

@@ -131,6 +131,8 @@ const char* fp8attn_status_string(int status) {
         case FP8ATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case FP8ATTN_ERR_CUDA: return "CUDA call failed";
         case FP8ATTN_ERR_TIMEOUT: return "device-side wait timed out";
+        case FP8ATTN_ERR_TOO_LARGE:
+            return "more heads than the built-in scratch of fp8attn_quantize_noalloc holds";
         default: return "unknown status";
     }
 }

@@ -9,6 +9,8 @@
 // head the maximum pass touched last, which is still in L2.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "common.h"
 
 namespace fp8attn {
@@ -149,3 +151,67 @@ int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
 }
 
 }  // namespace fp8attn
+
+// ---------------------------------------------------------------------------
+// Allocation-free variant of the quantizer.
+//
+// The per-head absmax accumulators normally live in the caller's workspace.
+// Here they live in a fixed array inside the library image, so a caller needs
+// nothing but its input and output buffers.
+// ---------------------------------------------------------------------------
+namespace fp8attn {
+namespace {
+
+constexpr int kStaticMaxHeads = FP8ATTN_NOALLOC_MAX_HEADS;
+
+// Resident on every GPU that loads the library, until the process exits.
+static __device__ __align__(256) uint32_t g_static_amax[kStaticMaxHeads];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+uint32_t* g_static_amax_addr[kMaxDevices] = {};
+
+// Device address of g_static_amax on the current device.  In host code the
+// symbol's name is only a handle, so the address is looked up once per device.
+int static_amax_address(uint32_t** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return FP8ATTN_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_amax_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_amax) != cudaSuccess || p == nullptr)
+            return FP8ATTN_ERR_CUDA;
+        g_static_amax_addr[dev] = static_cast<uint32_t*>(p);
+    }
+    *out = g_static_amax_addr[dev];
+    return FP8ATTN_OK;
+}
+
+}  // namespace
+}  // namespace fp8attn
+
+extern "C" int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int d,
+                                        const float* scale_in, void* x_fp8, float* scale_out,
+                                        void* cuda_stream) {
+    using namespace fp8attn;
+    if (B <= 0 || H <= 0 || rows < 0) return FP8ATTN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return FP8ATTN_ERR_UNSUPPORTED;
+    if ((int64_t)B * H > kStaticMaxHeads) return FP8ATTN_ERR_TOO_LARGE;
+    if (rows > 0 && (!x_bf16 || !x_fp8)) return FP8ATTN_ERR_INVALID_ARG;
+    if (!scale_in && !scale_out) return FP8ATTN_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(x_bf16) % 16 || reinterpret_cast<uintptr_t>(x_fp8) % 16 ||
+        reinterpret_cast<uintptr_t>(scale_in) % 4 || reinterpret_cast<uintptr_t>(scale_out) % 4)
+        return FP8ATTN_ERR_INVALID_ARG;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return FP8ATTN_ERR_CUDA;
+    if (major != 10) return FP8ATTN_ERR_UNSUPPORTED;
+    uint32_t* amax = nullptr;
+    int rc = static_amax_address(&amax);
+    if (rc != FP8ATTN_OK) return rc;
+    // launch_quantize clears the accumulators it uses at the start of every call
+    return launch_quantize(x_bf16, (int64_t)B * H, rows * (int64_t)d, scale_in, x_fp8, scale_out, amax,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
