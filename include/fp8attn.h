@@ -18,7 +18,9 @@
  *   - Return value: an fp8attn_status_t.  Argument errors are detected on the
  *     host before anything is launched.  Device-side problems (a bounded wait
  *     that ran out) are recorded in the workspace and read back with
- *     fp8attn_last_device_status(); the kernels never trap or spin forever.
+ *     fp8attn_last_device_status(); the kernels never trap or spin forever.  A
+ *     recorded device error is sticky: attention launches on that workspace do
+ *     nothing until fp8attn_last_device_status() has read and cleared it.
  *   - Supported head dims: d = 64 and d = 128.  n_train >= 1, n_test >= 0.
  */
 #ifndef FP8ATTN_H_

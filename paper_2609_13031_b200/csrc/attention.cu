@@ -1,16 +1,20 @@
 // Fused ICL attention for sm_100a: train->train and test->train in one launch.
 //
 // One CTA owns up to 256 query rows (two 128-row tiles) of one (b,h) and walks
-// over all train keys in tiles of 128.  Warp roles:
+// over all train keys in steps of kKeys keys.  Warp roles:
 //   warps 0-3  softmax of query tile 0 (one row per thread)
 //   warps 4-7  softmax of query tile 1
 //   warp  8    issues every tcgen05.mma (one elected thread)
 //   warp  9    TMA producer for Q, K and V tiles
-// Tensor memory (512 columns): S0 | S1 | O0 | O1.  The probability tile P_t is
-// written over the first columns of S_t (as e4m3 with the row maximum lifted to
-// 2^8, or as bf16 in the 16-bit path) and is the tensor-memory A operand of
-// O_t += P_t V.  While one tile's softmax runs on the CUDA cores, the tensor
-// core works on the other tile.
+//   warps 10-11 idle (they only give their registers to the softmax warps)
+// Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
+// thread pulls its whole score row into registers, releases S at once so that
+// the next Q K^T of its tile can run underneath the softmax, and writes the
+// probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 in the
+// 16-bit path) to its own tensor-memory region, from where it is the A operand
+// of O_t += P_t V.  Where 512 columns cannot hold a separate P (bf16, d = 128),
+// P is written over S and Q K^T waits for P V instead.  The FP8 d = 128 path
+// steps over 96 keys at a time to make room for P.
 //
 // Scale placement (FP8 path): x = (alpha * s_q * s_k * log2 e) * S feeds exp2;
 // the V scale and 1/rowsum are applied to O in the epilogue.
@@ -25,15 +29,18 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kTileM = 128;         // query rows per tile
-constexpr int kTileN = 128;         // keys per step
-constexpr int kNumThreads = 320;
+constexpr int kTileM = 128;           // query rows per tile
+constexpr int kNumThreads = 384;      // 8 softmax warps + MMA warp + TMA warp + 2 spare
+constexpr int kRegsSoftmax = 224;     // per-thread register budget after setmaxnreg
+constexpr int kRegsOther = 56;       // 8*32*224 + 4*32*56 leaves slack in the 64K register file:
+                                     // setmaxnreg.inc waits in hardware until the registers exist
 constexpr uint32_t kTmemCols = 512;
-constexpr uint64_t kWaitLimitNs = 4000000000ull;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 // detail codes written next to FP8ATTN_ERR_TIMEOUT
 enum : uint32_t {
-    kWaitQFull = 1, kWaitKFull, kWaitVFull, kWaitKEmpty, kWaitVEmpty, kWaitSFull, kWaitPFull, kWaitOFull
+    kWaitQFull = 1, kWaitKFull, kWaitVFull, kWaitKEmpty, kWaitVEmpty, kWaitSFull, kWaitPFull, kWaitOFull,
+    kWaitSFree, kWaitPFree
 };
 
 template <bool kFp8, int kD>
@@ -43,22 +50,30 @@ struct Cfg {
     static constexpr int kBoxBytes = kRowBytes > 128 ? 128 : kRowBytes;  // swizzle span
     static constexpr int kBoxes = kRowBytes / kBoxBytes;        // TMA boxes per tile
     static constexpr int kBoxCols = kBoxBytes / kES;
-    static constexpr int kTileBytes = 128 * kRowBytes;          // Q, K or V tile
+    static constexpr bool kSepP = !(kD == 128 && !kFp8);        // P in its own TMEM region
+    static constexpr int kKeys = (kFp8 && kD == 128) ? 96 : 128;  // keys per step
+    static constexpr int kQTileBytes = kTileM * kRowBytes;
+    static constexpr int kKVTileBytes = kKeys * kRowBytes;
     static constexpr int kUmmaK = 32 / kES;                     // elements per MMA K step
-    static constexpr int kStages = kTileBytes >= 32768 ? 2 : 4; // K ring and V ring depth
+    static constexpr int kStages = kKVTileBytes >= 32768 ? 2 : 4;  // K ring and V ring depth
     static constexpr uint32_t kSwizzle = kBoxBytes == 128 ? kSwizzle128 : kSwizzle64;
     static constexpr uint32_t kFmt = kFp8 ? 0u : 1u;            // e4m3 / bf16
-    static constexpr uint32_t kIdescQK = idesc(kFmt, kFmt, false, false, kTileM, kTileN);
+    static constexpr uint32_t kIdescQK = idesc(kFmt, kFmt, false, false, kTileM, kKeys);
     static constexpr uint32_t kIdescPV = idesc(kFmt, kFmt, false, true, kTileM, kD);
-    static constexpr uint32_t kColS = 0, kColO = 256;           // TMEM columns: S_t at t*128, O_t at 256+t*kD
-    static constexpr int kPCols = kTileN * kES / 4;             // TMEM columns of a P tile
-    static constexpr size_t kSmemBytes = (size_t)(2 + 2 * kStages) * kTileBytes + 1024;
+    static constexpr int kPCols = kKeys * kES / 4;              // TMEM columns of a P tile
+    // TMEM columns: S_t, then O_t at 256 + t*kD, P_t wherever 32-column-aligned room is left
+    static constexpr uint32_t kColS0 = 0, kColS1 = kKeys, kColO = 256;
+    static constexpr uint32_t kColP0 = !kSepP ? kColS0 : (kD == 128 ? 192u : 384u);
+    static constexpr uint32_t kColP1 = !kSepP ? kColS1 : (kD == 128 ? 224u : 384u + 64u);
+    static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
+    static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
+    static constexpr size_t kSmemBytes = (size_t)2 * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
 };
 
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_full[2];
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -79,6 +94,8 @@ struct Waiter {
         for (;;) {
             for (int i = 0; i < 64; ++i)
                 if (mbar_try_wait(bar, parity)) return true;
+            // another CTA already gave up: do not wait out the limit here as well
+            if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { dead = true; return false; }
             if (globaltimer_ns() - t0 > kWaitLimitNs) break;
         }
         dead = true;
@@ -105,6 +122,72 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
+// ---- packed fp32x2 arithmetic (two lanes per instruction on sm_100) ----
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// Blocks until this thread's tcgen05.ld results have landed; naming the 32
+// destination registers keeps every use of them after the wait.
+__device__ __forceinline__ void tmem_wait_ld_x32(uint32_t* r) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+                   "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]),
+                   "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]),
+                   "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                   "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]),
+                   "+r"(r[31])
+                 :
+                 : "memory");
+}
+
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
+#ifdef FP8ATTN_TRACE
+// Debug build only: clock stamps of CTA 0 (one lane per role) for a few steps.
+__device__ long long* g_trace_buf;
+#define FP8ATTN_TRACE_INIT() long long* const trace_buf = (blockIdx.x == 0) ? g_trace_buf : nullptr
+#define FP8ATTN_STAMP(slot, j)                                                         \
+    do {                                                                               \
+        if (trace_buf != nullptr && lane == 0 && (j) >= 64 && (j) < 80)                \
+            trace_buf[((j) - 64) * 32 + (slot)] = clock64();                           \
+    } while (0)
+#else
+#define FP8ATTN_TRACE_INIT() do { } while (0)
+#define FP8ATTN_STAMP(slot, j) do { } while (0)
+#endif
+
 struct KernelArgs {
     const float* scale_q; const float* scale_k; const float* scale_v;
     void* out_train; void* out_test;
@@ -121,6 +204,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                      const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const KernelArgs args) {
     using C = Cfg<kFp8, kD>;
+    constexpr int kKeys = C::kKeys;
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ uint32_t tmem_slot;
@@ -128,8 +212,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + 2 * C::kTileBytes;
-    const uint32_t sV = sK + C::kStages * C::kTileBytes;
+    const uint32_t sK = sQ + 2 * C::kQTileBytes;
+    const uint32_t sV = sK + C::kStages * C::kKVTileBytes;
 
     // ---- which query block is this CTA's ----
     const int blocks_per_head = args.blocks_train + args.blocks_test;
@@ -140,8 +224,12 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     const int64_t row0 = (int64_t)(is_test ? blk - args.blocks_train : blk) * (2 * kTileM);
     const int ntiles = (q_rows - row0 > kTileM) ? 2 : 1;
     const int64_t n_keys = args.n_train;
-    const int nkv = (int)((n_keys + kTileN - 1) / kTileN);
+    const int nkv = (int)((n_keys + kKeys - 1) / kKeys);
     const CUtensorMap* map_q = is_test ? &map_q_test : &map_q_train;
+
+    // A device error recorded earlier (and not yet read back by the host) is sticky:
+    // nothing runs until fp8attn_last_device_status() has cleared it.
+    if (*reinterpret_cast<volatile uint32_t*>(args.status) != 0u) return;
 
     // ---- set-up ----
     if (threadIdx.x == 0) {
@@ -154,7 +242,9 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.p_full[t]), kTileM);
+            mbar_init(smem_u32(&bars.s_free[t]), 4);
+            mbar_init(smem_u32(&bars.p_full[t]), 4);
+            mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
         }
         fence_mbar_init();
@@ -171,63 +261,87 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem = tmem_slot;
+    const uint32_t tmem = __shfl_sync(0xffffffffu, tmem_slot, 0);
     Waiter w{args.status, false};
+    FP8ATTN_TRACE_INIT();
 
-    if (warp == 9) {
+    if (warp >= 10) {
+        // spare warps: give up registers, then nothing to do until teardown
+        setmaxnreg_dec<kRegsOther>();
+    } else if (warp == 9) {
+        setmaxnreg_dec<kRegsOther>();
         // =========================== TMA producer ===========================
-        if (lane == 0) {
-            mbar_arrive_expect_tx(smem_u32(&bars.q_full), ntiles * C::kTileBytes);
+        // The whole warp walks the loop (waits included); one elected lane issues.
+        if (elect_one()) {
+            mbar_arrive_expect_tx(smem_u32(&bars.q_full), ntiles * C::kQTileBytes);
             for (int t = 0; t < ntiles; ++t)
                 for (int b = 0; b < C::kBoxes; ++b)
-                    tma_load_3d(sQ + t * C::kTileBytes + b * 128 * C::kBoxBytes, map_q,
+                    tma_load_3d(sQ + t * C::kQTileBytes + b * kTileM * C::kBoxBytes, map_q,
                                 b * C::kBoxCols, (int)(row0 + t * kTileM), bh,
                                 smem_u32(&bars.q_full));
-            for (int j = 0; j < nkv; ++j) {
-                const int s = j % C::kStages;
-                const uint32_t ph = (j / C::kStages) & 1;
-                w.wait(smem_u32(&bars.k_empty[s]), ph ^ 1, kWaitKEmpty);
-                mbar_arrive_expect_tx(smem_u32(&bars.k_full[s]), C::kTileBytes);
+        }
+        for (int j = 0; j < nkv; ++j) {
+            const int s = j % C::kStages;
+            const uint32_t ph = (j / C::kStages) & 1;
+            w.wait(smem_u32(&bars.k_empty[s]), ph ^ 1, kWaitKEmpty);
+            if (elect_one()) {
+                mbar_arrive_expect_tx(smem_u32(&bars.k_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
-                    tma_load_3d(sK + s * C::kTileBytes + b * 128 * C::kBoxBytes, &map_k,
-                                b * C::kBoxCols, j * kTileN, bh, smem_u32(&bars.k_full[s]));
-                w.wait(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
-                mbar_arrive_expect_tx(smem_u32(&bars.v_full[s]), C::kTileBytes);
-                for (int b = 0; b < C::kBoxes; ++b)
-                    tma_load_3d(sV + s * C::kTileBytes + b * 128 * C::kBoxBytes, &map_v,
-                                b * C::kBoxCols, j * kTileN, bh, smem_u32(&bars.v_full[s]));
+                    tma_load_3d(sK + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_k,
+                                b * C::kBoxCols, j * kKeys, bh, smem_u32(&bars.k_full[s]));
             }
-            if (w.dead) {
-                // let copies that are still in flight land before the CTA exits
-                Waiter d{args.status, false};
-                for (int j = (nkv > C::kStages ? nkv - C::kStages : 0); j < nkv; ++j) {
-                    d.wait(smem_u32(&bars.k_full[j % C::kStages]), (j / C::kStages) & 1, kWaitKFull);
-                    d.wait(smem_u32(&bars.v_full[j % C::kStages]), (j / C::kStages) & 1, kWaitVFull);
-                }
+            w.wait(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
+            if (elect_one()) {
+                mbar_arrive_expect_tx(smem_u32(&bars.v_full[s]), C::kKVTileBytes);
+                for (int b = 0; b < C::kBoxes; ++b)
+                    tma_load_3d(sV + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_v,
+                                b * C::kBoxCols, j * kKeys, bh, smem_u32(&bars.v_full[s]));
+            }
+            __syncwarp();
+        }
+        if (__any_sync(0xffffffffu, w.dead)) {
+            // let copies that are still in flight land before the CTA exits
+            Waiter d{args.status, false};
+            for (int j = (nkv > C::kStages ? nkv - C::kStages : 0); j < nkv; ++j) {
+                d.wait(smem_u32(&bars.k_full[j % C::kStages]), (j / C::kStages) & 1, kWaitKFull);
+                d.wait(smem_u32(&bars.v_full[j % C::kStages]), (j / C::kStages) & 1, kWaitVFull);
             }
         }
     } else if (warp == 8) {
+        setmaxnreg_dec<kRegsOther>();
         // ============================ MMA issuer ============================
-        if (lane == 0) {
+        // The whole warp walks the loop (waits included); one elected lane issues the
+        // MMAs and commits, so descriptor arithmetic stays on the uniform datapath.
+        {
+            // Descriptors are built once; per instruction only the 16-byte-unit start
+            // address in the low bits moves (all offsets are compile-time constants).
+            const uint64_t dQ = smem_desc(sQ, 0, 8 * C::kBoxBytes, C::kSwizzle);
+            const uint64_t dK = smem_desc(sK, 0, 8 * C::kBoxBytes, C::kSwizzle);
+            const uint64_t dV = smem_desc(sV, kKeys * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
+            auto commit_elected = [&](uint32_t bar) {
+                if (elect_one()) mma_commit(bar);
+            };
             auto issue_qk = [&](int t, int stage) {
+                const uint64_t a0 = dQ + (uint64_t)((t * C::kQTileBytes) >> 4);
+                const uint64_t b0 = dK + (uint64_t)((stage * C::kKVTileBytes) >> 4);
+                const uint32_t d = tmem + (t ? C::kColS1 : C::kColS0);
 #pragma unroll
                 for (int kk = 0; kk < kD / C::kUmmaK; ++kk) {
+                    constexpr int kB = C::kBoxBytes;
                     const int off = kk * 32;
-                    const uint32_t in_box = off % C::kBoxBytes, box = off / C::kBoxBytes;
-                    uint64_t a = smem_desc(sQ + t * C::kTileBytes + box * 128 * C::kBoxBytes + in_box,
-                                           0, 8 * C::kBoxBytes, C::kSwizzle);
-                    uint64_t b = smem_desc(sK + stage * C::kTileBytes + box * 128 * C::kBoxBytes + in_box,
-                                           0, 8 * C::kBoxBytes, C::kSwizzle);
-                    mma_ss<kFp8>(tmem + C::kColS + t * kTileN, a, b, C::kIdescQK, kk > 0);
+                    const uint64_t a = a0 + (uint64_t)(((off / kB) * kTileM * kB + off % kB) >> 4);
+                    const uint64_t b = b0 + (uint64_t)(((off / kB) * kKeys * kB + off % kB) >> 4);
+                    if (elect_one()) mma_ss<kFp8>(d, a, b, C::kIdescQK, kk > 0);
                 }
             };
             auto issue_pv = [&](int t, int stage, bool accumulate) {
+                const uint64_t b0 = dV + (uint64_t)((stage * C::kKVTileBytes) >> 4);
+                const uint32_t d = tmem + C::kColO + t * kD;
+                const uint32_t a = tmem + (t ? C::kColP1 : C::kColP0);
 #pragma unroll
-                for (int kk = 0; kk < kTileN / C::kUmmaK; ++kk) {
-                    uint64_t b = smem_desc(sV + stage * C::kTileBytes + kk * C::kUmmaK * C::kBoxBytes,
-                                           128 * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
-                    mma_ts<kFp8>(tmem + C::kColO + t * kD, tmem + C::kColS + t * kTileN + kk * 8, b,
-                                 C::kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < kKeys / C::kUmmaK; ++kk) {
+                    const uint64_t b = b0 + (uint64_t)((kk * C::kUmmaK * C::kBoxBytes) >> 4);
+                    if (elect_one()) mma_ts<kFp8>(d, a + kk * 8, b, C::kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
                 }
             };
             w.wait(smem_u32(&bars.q_full), 0, kWaitQFull);
@@ -235,36 +349,92 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             tc_fence_after_sync();
             for (int t = 0; t < ntiles; ++t) {
                 issue_qk(t, 0);
-                mma_commit(smem_u32(&bars.s_full[t]));
+                commit_elected(smem_u32(&bars.s_full[t]));
             }
-            mma_commit(smem_u32(&bars.k_empty[0]));
-            for (int j = 0; j < nkv; ++j) {
-                const int sv = j % C::kStages;
-                const bool has_next = j + 1 < nkv;
-                const int sk = (j + 1) % C::kStages;
-                w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
-                if (has_next) w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
-                for (int t = 0; t < ntiles; ++t) {
-                    w.wait(smem_u32(&bars.p_full[t]), j & 1, kWaitPFull);
+            commit_elected(smem_u32(&bars.k_empty[0]));
+            if (C::kSepP) {
+                // Event order per step: Q K^T(j+1) of tile 0, P V(j-1) of tile 1, Q K^T(j+1)
+                // of tile 1, P V(j) of tile 0.  It keeps the two tiles half a step apart, so
+                // one tile's exponentials run while the other waits for tensor memory.
+                auto pv_tile1 = [&](int jj) {
+                    const int st = jj % C::kStages;
+                    w.wait(smem_u32(&bars.p_full[1]), jj & 1, kWaitPFull);
                     tc_fence_after_sync();
-                    issue_pv(t, sv, j > 0);
-                    if (!has_next) mma_commit(smem_u32(&bars.o_full[t]));
+                    FP8ATTN_STAMP(18, jj);
+                    issue_pv(1, st, jj > 0);
+                    commit_elected(smem_u32(&bars.p_free[1]));
+                    if (jj + 1 == nkv) commit_elected(smem_u32(&bars.o_full[1]));
+                    commit_elected(smem_u32(&bars.v_empty[st]));
+                    FP8ATTN_STAMP(19, jj);
+                };
+                for (int j = 0; j < nkv; ++j) {
+                    const int sv = j % C::kStages;
+                    const bool has_next = j + 1 < nkv;
+                    const int sk = (j + 1) % C::kStages;
                     if (has_next) {
-                        issue_qk(t, sk);
-                        mma_commit(smem_u32(&bars.s_full[t]));
+                        w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
+                        w.wait(smem_u32(&bars.s_free[0]), j & 1, kWaitSFree);
+                        tc_fence_after_sync();
+                        FP8ATTN_STAMP(20, j);
+                        issue_qk(0, sk);
+                        commit_elected(smem_u32(&bars.s_full[0]));
                     }
+                    if (ntiles == 2 && j > 0) pv_tile1(j - 1);
+                    if (has_next) {
+                        if (ntiles == 2) {
+                            w.wait(smem_u32(&bars.s_free[1]), j & 1, kWaitSFree);
+                            tc_fence_after_sync();
+                            FP8ATTN_STAMP(21, j);
+                            issue_qk(1, sk);
+                            commit_elected(smem_u32(&bars.s_full[1]));
+                        }
+                        commit_elected(smem_u32(&bars.k_empty[sk]));
+                    }
+                    w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
+                    w.wait(smem_u32(&bars.p_full[0]), j & 1, kWaitPFull);
+                    tc_fence_after_sync();
+                    FP8ATTN_STAMP(16, j);
+                    issue_pv(0, sv, j > 0);
+                    commit_elected(smem_u32(&bars.p_free[0]));
+                    if (!has_next) commit_elected(smem_u32(&bars.o_full[0]));
+                    if (ntiles == 1) commit_elected(smem_u32(&bars.v_empty[sv]));
+                    FP8ATTN_STAMP(17, j);
                 }
-                mma_commit(smem_u32(&bars.v_empty[sv]));
-                if (has_next) mma_commit(smem_u32(&bars.k_empty[sk]));
+                if (ntiles == 2) pv_tile1(nkv - 1);
+            } else {
+                // P lives in S: P V(j) then Q K^T(j+1) per tile, which overwrites that P
+                for (int j = 0; j < nkv; ++j) {
+                    const int sv = j % C::kStages;
+                    const bool has_next = j + 1 < nkv;
+                    const int sk = (j + 1) % C::kStages;
+                    w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
+                    if (has_next) w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
+                    for (int t = 0; t < ntiles; ++t) {
+                        w.wait(smem_u32(&bars.p_full[t]), j & 1, kWaitPFull);
+                        tc_fence_after_sync();
+                        FP8ATTN_STAMP(16 + t * 2, j);
+                        issue_pv(t, sv, j > 0);
+                        if (!has_next) commit_elected(smem_u32(&bars.o_full[t]));
+                        if (has_next) {
+                            issue_qk(t, sk);
+                            commit_elected(smem_u32(&bars.s_full[t]));
+                        }
+                        FP8ATTN_STAMP(17 + t * 2, j);
+                    }
+                    commit_elected(smem_u32(&bars.v_empty[sv]));
+                    if (has_next) commit_elected(smem_u32(&bars.k_empty[sk]));
+                }
             }
         }
     } else {
         // ========================= softmax + epilogue =========================
+        setmaxnreg_inc<kRegsSoftmax>();
         const int t = warp >> 2;                 // query tile of this warpgroup
         if (t < ntiles) {
             const int row_in_tile = threadIdx.x & 127;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + lane_addr + C::kColS + t * kTileN;
+            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0);
+            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0);
             const uint32_t tO = tmem + lane_addr + C::kColO + t * kD;
             float c = (args.softmax_scale > 0.f ? args.softmax_scale : rsqrtf((float)kD)) *
                       1.4426950408889634f;
@@ -274,64 +444,110 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 sv_scale = args.scale_v[bh];
             }
             const float lift = kFp8 ? 8.0f : 0.0f;
-            float m = -INFINITY, l = 0.f;
+            const uint64_t cc = pack2(c, c);
+            float m = -INFINITY;
+            uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // four partial row sums
+            constexpr uint32_t kNegInf = 0xff800000u;
             for (int j = 0; j < nkv; ++j) {
                 w.wait(smem_u32(&bars.s_full[t]), j & 1, kWaitSFull);
                 tc_fence_after_sync();
-                float s[kTileN];
+                FP8ATTN_STAMP(t * 8 + 0, j);
+                // ---- the whole score row of this thread into registers ----
+                uint32_t s[kKeys];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) tmem_ld_x32(tS + q * 32, reinterpret_cast<uint32_t*>(s) + q * 32);
-                tmem_wait_ld();
-                const int valid = (int)min((int64_t)kTileN, n_keys - (int64_t)j * kTileN);
-                if (valid < kTileN) {
+                for (int q = 0; q < kKeys / 32; ++q) tmem_ld_x32(tS + q * 32, s + q * 32);
 #pragma unroll
-                    for (int i = 0; i < kTileN; ++i)
-                        if (i >= valid) s[i] = -INFINITY;
+                for (int q = 0; q < kKeys / 32; ++q) tmem_wait_ld_x32(s + q * 32);
+                if (C::kSepP) {
+                    // S may be overwritten by the next Q K^T from here on
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
                 }
-                float mx = s[0];
+                FP8ATTN_STAMP(t * 8 + 1, j);
+                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys);
+                if (valid < kKeys) {
 #pragma unroll
-                for (int i = 1; i < kTileN; ++i) mx = fmaxf(mx, s[i]);
-                const float m_new = fmaxf(m, mx);
+                    for (int i = 0; i < kKeys; ++i)
+                        if (i >= valid) s[i] = kNegInf;
+                }
+                // ---- row maximum of the raw scores ----
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < kKeys; i += 8) {
+                    mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+                    mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+                    mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+                    mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+                }
+                const float m_new = max3(m, fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                // P V of the previous step must be done before O is rescaled or P rewritten
+                bool pv_done = !(C::kSepP && j > 0);
                 if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
+                    if (!pv_done) {
+                        w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                        tc_fence_after_sync();
+                        pv_done = true;
+                    }
                     // the running maximum moved for some row of this warp: rescale O and l
                     const float f = ex2((m - m_new) * c);
-                    l *= f;
+                    const uint64_t ff = pack2(f, f);
+                    l2a = mul2(l2a, ff);
+                    l2b = mul2(l2b, ff);
 #pragma unroll
                     for (int q = 0; q < kD / 32; ++q) {
-                        float o[32];
-                        tmem_ld_x32(tO + q * 32, reinterpret_cast<uint32_t*>(o));
-                        tmem_wait_ld();
+                        uint32_t o[32];
+                        tmem_ld_x32(tO + q * 32, o);
+                        tmem_wait_ld_x32(o);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= f;
-                        tmem_st_x32(tO + q * 32, reinterpret_cast<uint32_t*>(o));
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st_x32(tO + q * 32, o);
                     }
                 }
                 m = m_new;
                 const float nb = lift - m * c;
-                float sum = 0.f;
-                uint32_t p[C::kPCols];
-                if (kFp8) {
+                const uint64_t nbnb = pack2(nb, nb);
+                FP8ATTN_STAMP(t * 8 + 2, j);
+                // ---- p = 2^(c*s - c*m + lift), row sums, P tile into tensor memory ----
 #pragma unroll
-                    for (int i = 0; i < kTileN; i += 4) {
-                        float p0 = ex2(fmaf(s[i], c, nb)), p1 = ex2(fmaf(s[i + 1], c, nb));
-                        float p2 = ex2(fmaf(s[i + 2], c, nb)), p3 = ex2(fmaf(s[i + 3], c, nb));
-                        sum += (p0 + p1) + (p2 + p3);
-                        p[i / 4] = pack_e4m3x4(p0, p1, p2, p3);
-                    }
-                } else {
+                for (int q = 0; q < kKeys / 32; ++q) {
+                    uint32_t p[kFp8 ? 8 : 16];
 #pragma unroll
-                    for (int i = 0; i < kTileN; i += 2) {
-                        float p0 = ex2(fmaf(s[i], c, nb)), p1 = ex2(fmaf(s[i + 1], c, nb));
-                        sum += p0 + p1;
-                        p[i / 2] = pack_bf16x2(p0, p1);
+                    for (int i = 0; i < 32; i += 4) {
+                        const uint32_t* cur = s + q * 32 + i;
+                        float x0, x1, x2, x3;
+                        unpack2(fma2(pack2(__uint_as_float(cur[0]), __uint_as_float(cur[1])), cc, nbnb), x0, x1);
+                        unpack2(fma2(pack2(__uint_as_float(cur[2]), __uint_as_float(cur[3])), cc, nbnb), x2, x3);
+                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                        l2a = add2(l2a, pack2(p0, p1));
+                        l2b = add2(l2b, pack2(p2, p3));
+                        if (kFp8) {
+                            p[i / 4] = pack_e4m3x4(p0, p1, p2, p3);
+                        } else {
+                            p[i / 2] = pack_bf16x2(p0, p1);
+                            p[i / 2 + 1] = pack_bf16x2(p2, p3);
+                        }
                     }
+                    if (q == 0 && !pv_done) {
+                        w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                        tc_fence_after_sync();
+                    }
+                    if (kFp8) tmem_st_x8(tP + q * 8, p);
+                    else tmem_st_x16(tP + q * 16, p);
                 }
-                l += sum;
-#pragma unroll
-                for (int q = 0; q < C::kPCols / 32; ++q) tmem_st_x32(tS + q * 32, p + q * 32);
+                FP8ATTN_STAMP(t * 8 + 3, j);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(smem_u32(&bars.p_full[t]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
+                FP8ATTN_STAMP(t * 8 + 4, j);
+            }
+            float l;
+            {
+                float a0, a1, b0, b1;
+                unpack2(l2a, a0, a1);
+                unpack2(l2b, b0, b1);
+                l = (a0 + a1) + (b0 + b1);
             }
             // ---- epilogue: out = s_v * O / l ----
             w.wait(smem_u32(&bars.o_full[t]), 0, kWaitOFull);
@@ -342,17 +558,17 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                                  ((int64_t)bh * q_rows + row) * kD;
 #pragma unroll
             for (int q = 0; q < kD / 32; ++q) {
-                float o[32];
-                tmem_ld_x32(tO + q * 32, reinterpret_cast<uint32_t*>(o));
-                tmem_wait_ld();
+                uint32_t o[32];
+                tmem_ld_x32(tO + q * 32, o);
+                tmem_wait_ld_x32(o);
                 if (row < q_rows && !w.dead) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint4 v;
-                        v.x = pack_bf16x2(o[i] * inv, o[i + 1] * inv);
-                        v.y = pack_bf16x2(o[i + 2] * inv, o[i + 3] * inv);
-                        v.z = pack_bf16x2(o[i + 4] * inv, o[i + 5] * inv);
-                        v.w = pack_bf16x2(o[i + 6] * inv, o[i + 7] * inv);
+                        v.x = pack_bf16x2(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
                         *reinterpret_cast<uint4*>(out + q * 32 + i) = v;
                     }
                 }
@@ -371,8 +587,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     const int64_t heads = (int64_t)p.B * p.H;
     CUtensorMap mq_train, mq_test, mk, mv;
     if (!make_tensor_map(&mq_train, p.q_train, C::kES, heads, p.n_train, kD, kTileM, C::kBoxCols) ||
-        !make_tensor_map(&mk, p.k, C::kES, heads, p.n_train, kD, kTileN, C::kBoxCols) ||
-        !make_tensor_map(&mv, p.v, C::kES, heads, p.n_train, kD, kTileN, C::kBoxCols))
+        !make_tensor_map(&mk, p.k, C::kES, heads, p.n_train, kD, C::kKeys, C::kBoxCols) ||
+        !make_tensor_map(&mv, p.v, C::kES, heads, p.n_train, kD, C::kKeys, C::kBoxCols))
         return FP8ATTN_ERR_CUDA;
     if (p.n_test > 0) {
         if (!make_tensor_map(&mq_test, p.q_test, C::kES, heads, p.n_test, kD, kTileM, C::kBoxCols))
@@ -404,6 +620,15 @@ int launch(const AttnParams& p, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef FP8ATTN_TRACE
+// Debug build only: where the kernels of CTA 0 write their clock stamps
+// (16 steps x 32 slots of int64), or NULL to switch tracing off.
+extern "C" int fp8attn_debug_set_trace(void* device_buffer) {
+    long long* p = static_cast<long long*>(device_buffer);
+    return cudaMemcpyToSymbol(g_trace_buf, &p, sizeof(p)) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {
     if (fp8) return p.d == 64 ? launch<true, 64>(p, stream) : launch<true, 128>(p, stream);
