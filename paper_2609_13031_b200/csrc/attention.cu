@@ -2,11 +2,15 @@
 //
 // One CTA owns up to 256 query rows (two 128-row tiles) of one (b,h) and walks
 // over all train keys in steps of kKeys keys.  Warp roles:
-//   warps 0-3  softmax of query tile 0 (one row per thread)
-//   warps 4-7  softmax of query tile 1
-//   warp  8    issues every tcgen05.mma (one elected thread)
-//   warp  9    TMA producer for Q, K and V tiles
-//   warps 10-11 idle (they only give their registers to the softmax warps)
+//   warps 0-7   softmax of query tile 0: two threads per row, each owning half of
+//               the key columns of a step (warps 0-3: first half, 4-7: second half)
+//   warps 8-15  softmax of query tile 1, same split
+//   warp  16    issues the Q K^T tcgen05.mma of both tiles (one elected lane)
+//   warp  17    TMA producer for Q, K and V tiles
+//   warps 18-19 issue the P V tcgen05.mma of tile 0 and tile 1
+// Four softmax warps per scheduler hide each other's tensor-memory, MUFU and
+// barrier latencies; the two threads of a row exchange their partial maxima
+// through shared memory once per step.
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
@@ -30,10 +34,19 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileM = 128;           // query rows per tile
-constexpr int kNumThreads = 384;      // 8 softmax warps + MMA warp + TMA warp + 2 spare
-constexpr int kRegsSoftmax = 224;     // per-thread register budget after setmaxnreg
-constexpr int kRegsOther = 56;       // 8*32*224 + 4*32*56 leaves slack in the 64K register file:
-                                     // setmaxnreg.inc waits in hardware until the registers exist
+#ifndef FP8ATTN_POLY_EVERY
+#define FP8ATTN_POLY_EVERY 2
+#endif
+constexpr int kSoftmaxWarps = 16;
+constexpr int kQkWarp = 16, kTmaWarp = 17, kPvWarp0 = 18;   // warps 18, 19: P V of tile 0, 1
+constexpr int kNumThreads = 640;      // 16 softmax warps + MMA warp + TMA warp + 2 spare
+// Register budgets after setmaxnreg.  The CTA's register pool is what it was
+// launched with (640 threads x 96); setmaxnreg.inc waits in hardware until the pool
+// can serve it, so the budgets must fit: 16*32*104 + 4*32*56 = 60416 <= 61440.
+constexpr int kRegsSoftmax = 104;
+constexpr int kRegsOther = 56;
+static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + (kNumThreads - kSoftmaxWarps * 32) * kRegsOther <=
+                  kNumThreads * 96, "setmaxnreg budgets exceed the CTA's register pool");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
@@ -111,10 +124,16 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 __device__ __forceinline__ uint32_t pack_e4m3x4(float a, float b, float c, float d) {
-    uint16_t lo, hi;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(b), "f"(a));
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(d), "f"(c));
-    return (uint32_t)lo | ((uint32_t)hi << 16);
+    uint32_t r;
+    asm("{\n"
+        ".reg .b16 lo, hi;\n"
+        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n"
+        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n"
+        "mov.b32 %0, {lo, hi};\n"
+        "}\n"
+        : "=r"(r)
+        : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
@@ -151,8 +170,48 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
+// 2^x for a pair of lanes on the FMA pipe instead of the MUFU: x = n + f with
+// n = round(x) taken from the mantissa after adding 1.5*2^23, f in [-0.5, 0.5],
+// 2^f by a minimax polynomial (degree 2: 1.7e-3 relative, enough for an e4m3
+// result; degree 3: 7.5e-5 for bf16), and n added into the exponent field.
+// x must be >= -126 (the caller clamps) and < 128.
+template <bool kDegree3>
+__device__ __forceinline__ void exp2_poly2(uint64_t x, float& r0, float& r1) {
+    const uint64_t magic = pack2(12582912.f, 12582912.f);
+    const uint64_t neg_magic = pack2(-12582912.f, -12582912.f);
+    const uint64_t neg_one = pack2(-1.f, -1.f);
+    const uint64_t t = add2(x, magic);
+    const uint64_t n = add2(t, neg_magic);
+    const uint64_t f = fma2(n, neg_one, x);
+    uint64_t p;
+    if (kDegree3) {
+        p = fma2(f, pack2(0.05517132f, 0.05517132f), pack2(0.24261054f, 0.24261054f));
+        p = fma2(p, f, pack2(0.69326097f, 0.69326097f));
+        p = fma2(p, f, pack2(0.99992812f, 0.99992812f));
+    } else {
+        p = fma2(f, pack2(0.23842570f, 0.23842570f), pack2(0.70344281f, 0.70344281f));
+        p = fma2(p, f, pack2(1.00044298f, 1.00044298f));
+    }
+    float p0, p1, t0, t1;
+    unpack2(p, p0, p1);
+    unpack2(t, t0, t1);
+    r0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    r1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
 // Blocks until this thread's tcgen05.ld results have landed; naming the 32
 // destination registers keeps every use of them after the wait.
+__device__ __forceinline__ void tmem_wait_ld_x16(uint32_t* r) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+                   "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]),
+                   "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld_x32(uint32_t* r) {
     asm volatile("tcgen05.wait::ld.sync.aligned;"
                  : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
@@ -180,7 +239,7 @@ __device__ long long* g_trace_buf;
 #define FP8ATTN_TRACE_INIT() long long* const trace_buf = (blockIdx.x == 0) ? g_trace_buf : nullptr
 #define FP8ATTN_STAMP(slot, j)                                                         \
     do {                                                                               \
-        if (trace_buf != nullptr && lane == 0 && (j) >= 64 && (j) < 80)                \
+        if (trace_buf != nullptr && lane == 0 && (warp >= 16 || (warp & 7) == 0) && (j) >= 64 && (j) < 80)                \
             trace_buf[((j) - 64) * 32 + (slot)] = clock64();                           \
     } while (0)
 #else
@@ -208,6 +267,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ uint32_t tmem_slot;
+    __shared__ float xchg[2][2][2][kTileM];   // [step parity][tile][column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -238,12 +298,12 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             mbar_init(smem_u32(&bars.k_full[s]), 1);
             mbar_init(smem_u32(&bars.k_empty[s]), 1);
             mbar_init(smem_u32(&bars.v_full[s]), 1);
-            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), ntiles);   // one commit per P V issuer
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.s_free[t]), 4);
-            mbar_init(smem_u32(&bars.p_full[t]), 4);
+            mbar_init(smem_u32(&bars.s_free[t]), 8);
+            mbar_init(smem_u32(&bars.p_full[t]), 8);
             mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
         }
@@ -253,7 +313,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
-    if (warp == 9 && lane == 0) {
+    if (warp == kTmaWarp && lane == 0) {
         prefetch_tensormap(map_q);
         prefetch_tensormap(&map_k);
         prefetch_tensormap(&map_v);
@@ -265,10 +325,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     Waiter w{args.status, false};
     FP8ATTN_TRACE_INIT();
 
-    if (warp >= 10) {
-        // spare warps: give up registers, then nothing to do until teardown
-        setmaxnreg_dec<kRegsOther>();
-    } else if (warp == 9) {
+    if (warp == kTmaWarp) {
         setmaxnreg_dec<kRegsOther>();
         // =========================== TMA producer ===========================
         // The whole warp walks the loop (waits included); one elected lane issues.
@@ -307,135 +364,98 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 d.wait(smem_u32(&bars.v_full[j % C::kStages]), (j / C::kStages) & 1, kWaitVFull);
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == kQkWarp) {
         setmaxnreg_dec<kRegsOther>();
-        // ============================ MMA issuer ============================
+        // ====================== Q K^T issuer (both query tiles) ======================
         // The whole warp walks the loop (waits included); one elected lane issues the
-        // MMAs and commits, so descriptor arithmetic stays on the uniform datapath.
-        {
-            // Descriptors are built once; per instruction only the 16-byte-unit start
-            // address in the low bits moves (all offsets are compile-time constants).
-            const uint64_t dQ = smem_desc(sQ, 0, 8 * C::kBoxBytes, C::kSwizzle);
-            const uint64_t dK = smem_desc(sK, 0, 8 * C::kBoxBytes, C::kSwizzle);
-            const uint64_t dV = smem_desc(sV, kKeys * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
-            auto commit_elected = [&](uint32_t bar) {
-                if (elect_one()) mma_commit(bar);
-            };
-            auto issue_qk = [&](int t, int stage) {
-                const uint64_t a0 = dQ + (uint64_t)((t * C::kQTileBytes) >> 4);
-                const uint64_t b0 = dK + (uint64_t)((stage * C::kKVTileBytes) >> 4);
-                const uint32_t d = tmem + (t ? C::kColS1 : C::kColS0);
+        // MMAs and commits.  Q K^T and P V are issued from different warps because one
+        // warp cannot issue tcgen05 instructions fast enough to feed the tensor core
+        // with instructions of this size; every dependency between the two streams
+        // already goes through an mbarrier.
+        const uint64_t dQ = smem_desc(sQ, 0, 8 * C::kBoxBytes, C::kSwizzle);
+        const uint64_t dK = smem_desc(sK, 0, 8 * C::kBoxBytes, C::kSwizzle);
+        auto issue_qk = [&](int t, int stage) {
+            const uint64_t a0 = dQ + (uint64_t)((t * C::kQTileBytes) >> 4);
+            const uint64_t b0 = dK + (uint64_t)((stage * C::kKVTileBytes) >> 4);
+            const uint32_t d = tmem + (t ? C::kColS1 : C::kColS0);
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kD / C::kUmmaK; ++kk) {
                     constexpr int kB = C::kBoxBytes;
                     const int off = kk * 32;
                     const uint64_t a = a0 + (uint64_t)(((off / kB) * kTileM * kB + off % kB) >> 4);
                     const uint64_t b = b0 + (uint64_t)(((off / kB) * kKeys * kB + off % kB) >> 4);
-                    if (elect_one()) mma_ss<kFp8>(d, a, b, C::kIdescQK, kk > 0);
+                    mma_ss<kFp8>(d, a, b, C::kIdescQK, kk > 0);
                 }
-            };
-            auto issue_pv = [&](int t, int stage, bool accumulate) {
-                const uint64_t b0 = dV + (uint64_t)((stage * C::kKVTileBytes) >> 4);
-                const uint32_t d = tmem + C::kColO + t * kD;
-                const uint32_t a = tmem + (t ? C::kColP1 : C::kColP0);
-#pragma unroll
-                for (int kk = 0; kk < kKeys / C::kUmmaK; ++kk) {
-                    const uint64_t b = b0 + (uint64_t)((kk * C::kUmmaK * C::kBoxBytes) >> 4);
-                    if (elect_one()) mma_ts<kFp8>(d, a + kk * 8, b, C::kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
-                }
-            };
-            w.wait(smem_u32(&bars.q_full), 0, kWaitQFull);
-            w.wait(smem_u32(&bars.k_full[0]), 0, kWaitKFull);
-            tc_fence_after_sync();
-            for (int t = 0; t < ntiles; ++t) {
-                issue_qk(t, 0);
-                commit_elected(smem_u32(&bars.s_full[t]));
+                mma_commit(smem_u32(&bars.s_full[t]));
             }
-            commit_elected(smem_u32(&bars.k_empty[0]));
-            if (C::kSepP) {
-                // Event order per step: Q K^T(j+1) of tile 0, P V(j-1) of tile 1, Q K^T(j+1)
-                // of tile 1, P V(j) of tile 0.  It keeps the two tiles half a step apart, so
-                // one tile's exponentials run while the other waits for tensor memory.
-                auto pv_tile1 = [&](int jj) {
-                    const int st = jj % C::kStages;
-                    w.wait(smem_u32(&bars.p_full[1]), jj & 1, kWaitPFull);
-                    tc_fence_after_sync();
-                    FP8ATTN_STAMP(18, jj);
-                    issue_pv(1, st, jj > 0);
-                    commit_elected(smem_u32(&bars.p_free[1]));
-                    if (jj + 1 == nkv) commit_elected(smem_u32(&bars.o_full[1]));
-                    commit_elected(smem_u32(&bars.v_empty[st]));
-                    FP8ATTN_STAMP(19, jj);
-                };
-                for (int j = 0; j < nkv; ++j) {
-                    const int sv = j % C::kStages;
-                    const bool has_next = j + 1 < nkv;
-                    const int sk = (j + 1) % C::kStages;
-                    if (has_next) {
-                        w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
-                        w.wait(smem_u32(&bars.s_free[0]), j & 1, kWaitSFree);
-                        tc_fence_after_sync();
-                        FP8ATTN_STAMP(20, j);
-                        issue_qk(0, sk);
-                        commit_elected(smem_u32(&bars.s_full[0]));
+            __syncwarp();
+        };
+        w.wait(smem_u32(&bars.q_full), 0, kWaitQFull);
+        w.wait(smem_u32(&bars.k_full[0]), 0, kWaitKFull);
+        tc_fence_after_sync();
+        for (int t = 0; t < ntiles; ++t) issue_qk(t, 0);
+        if (elect_one()) mma_commit(smem_u32(&bars.k_empty[0]));
+        __syncwarp();
+        for (int j = 0; j + 1 < nkv; ++j) {
+            const int sk = (j + 1) % C::kStages;
+            w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
+            for (int t = 0; t < ntiles; ++t) {
+                // S_t is free once its rows sit in registers; where P is written over S,
+                // only once P V of this step has consumed it
+                if (C::kSepP) w.wait(smem_u32(&bars.s_free[t]), j & 1, kWaitSFree);
+                else w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
+                tc_fence_after_sync();
+                FP8ATTN_STAMP(20 + t, j);
+                issue_qk(t, sk);
+            }
+            if (elect_one()) mma_commit(smem_u32(&bars.k_empty[sk]));
+            __syncwarp();
+        }
+    } else if (warp >= kPvWarp0) {
+        setmaxnreg_dec<kRegsOther>();
+        // ========================= P V issuer of one query tile =========================
+        const int t = warp - kPvWarp0;
+        if (t < ntiles) {
+            const uint64_t dV = smem_desc(sV, kKeys * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
+            const uint32_t d = tmem + C::kColO + t * kD;
+            const uint32_t a = tmem + (t ? C::kColP1 : C::kColP0);
+            for (int j = 0; j < nkv; ++j) {
+                const int sv = j % C::kStages;
+                w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
+                w.wait(smem_u32(&bars.p_full[t]), j & 1, kWaitPFull);
+                tc_fence_after_sync();
+                FP8ATTN_STAMP(16 + t * 2, j);
+                if (elect_one()) {
+                    const uint64_t b0 = dV + (uint64_t)((sv * C::kKVTileBytes) >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < kKeys / C::kUmmaK; ++kk) {
+                        const uint64_t b = b0 + (uint64_t)((kk * C::kUmmaK * C::kBoxBytes) >> 4);
+                        mma_ts<kFp8>(d, a + kk * 8, b, C::kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
                     }
-                    if (ntiles == 2 && j > 0) pv_tile1(j - 1);
-                    if (has_next) {
-                        if (ntiles == 2) {
-                            w.wait(smem_u32(&bars.s_free[1]), j & 1, kWaitSFree);
-                            tc_fence_after_sync();
-                            FP8ATTN_STAMP(21, j);
-                            issue_qk(1, sk);
-                            commit_elected(smem_u32(&bars.s_full[1]));
-                        }
-                        commit_elected(smem_u32(&bars.k_empty[sk]));
-                    }
-                    w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
-                    w.wait(smem_u32(&bars.p_full[0]), j & 1, kWaitPFull);
-                    tc_fence_after_sync();
-                    FP8ATTN_STAMP(16, j);
-                    issue_pv(0, sv, j > 0);
-                    commit_elected(smem_u32(&bars.p_free[0]));
-                    if (!has_next) commit_elected(smem_u32(&bars.o_full[0]));
-                    if (ntiles == 1) commit_elected(smem_u32(&bars.v_empty[sv]));
-                    FP8ATTN_STAMP(17, j);
+                    mma_commit(smem_u32(&bars.p_free[t]));
+                    mma_commit(smem_u32(&bars.v_empty[sv]));
+                    if (j + 1 == nkv) mma_commit(smem_u32(&bars.o_full[t]));
                 }
-                if (ntiles == 2) pv_tile1(nkv - 1);
-            } else {
-                // P lives in S: P V(j) then Q K^T(j+1) per tile, which overwrites that P
-                for (int j = 0; j < nkv; ++j) {
-                    const int sv = j % C::kStages;
-                    const bool has_next = j + 1 < nkv;
-                    const int sk = (j + 1) % C::kStages;
-                    w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
-                    if (has_next) w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
-                    for (int t = 0; t < ntiles; ++t) {
-                        w.wait(smem_u32(&bars.p_full[t]), j & 1, kWaitPFull);
-                        tc_fence_after_sync();
-                        FP8ATTN_STAMP(16 + t * 2, j);
-                        issue_pv(t, sv, j > 0);
-                        if (!has_next) commit_elected(smem_u32(&bars.o_full[t]));
-                        if (has_next) {
-                            issue_qk(t, sk);
-                            commit_elected(smem_u32(&bars.s_full[t]));
-                        }
-                        FP8ATTN_STAMP(17 + t * 2, j);
-                    }
-                    commit_elected(smem_u32(&bars.v_empty[sv]));
-                    if (has_next) commit_elected(smem_u32(&bars.k_empty[sk]));
-                }
+                __syncwarp();
+                FP8ATTN_STAMP(17 + t * 2, j);
             }
         }
     } else {
         // ========================= softmax + epilogue =========================
         setmaxnreg_inc<kRegsSoftmax>();
-        const int t = warp >> 2;                 // query tile of this warpgroup
+        constexpr int kHalf = kKeys / 2;         // key columns of a step owned by one thread
+        constexpr int kPHalf = C::kPCols / 2;    // P columns owned by one thread
+        constexpr int kOHalf = kD / 2;           // output columns owned by one thread
+        const int t = warp >> 3;                 // query tile
+        const int h = (warp >> 2) & 1;           // column half
         if (t < ntiles) {
-            const int row_in_tile = threadIdx.x & 127;
+            const int row_in_tile = (warp & 3) * 32 + lane;
+            const uint32_t pair_barrier = 1 + t * 4 + (warp & 3);   // the two warps that share rows
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0);
-            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0);
-            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD;
+            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0) + h * kHalf;
+            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0) + h * kPHalf;
+            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD + h * kOHalf;
             float c = (args.softmax_scale > 0.f ? args.softmax_scale : rsqrtf((float)kD)) *
                       1.4426950408889634f;
             float sv_scale = 1.0f;
@@ -444,20 +464,24 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 sv_scale = args.scale_v[bh];
             }
             const float lift = kFp8 ? 8.0f : 0.0f;
+            // every kPolyEvery-th group of four columns computes two of its exponentials
+            // with the polynomial (0 = never): 1 -> 50 %, 2 -> 25 %, 4 -> 12.5 % of all
+            constexpr int kPolyEvery = FP8ATTN_POLY_EVERY;
+            constexpr float kSlack = 0.0f;   // exact running maximum: the row maximum maps to 2^lift
             const uint64_t cc = pack2(c, c);
             float m = -INFINITY;
-            uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // four partial row sums
+            uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // partial row sums of this half
             constexpr uint32_t kNegInf = 0xff800000u;
             for (int j = 0; j < nkv; ++j) {
                 w.wait(smem_u32(&bars.s_full[t]), j & 1, kWaitSFull);
                 tc_fence_after_sync();
                 FP8ATTN_STAMP(t * 8 + 0, j);
-                // ---- the whole score row of this thread into registers ----
-                uint32_t s[kKeys];
+                // ---- this thread's half of the score row into registers ----
+                uint32_t s[kHalf];
 #pragma unroll
-                for (int q = 0; q < kKeys / 32; ++q) tmem_ld_x32(tS + q * 32, s + q * 32);
+                for (int q = 0; q < kHalf / 16; ++q) tmem_ld_x16(tS + q * 16, s + q * 16);
 #pragma unroll
-                for (int q = 0; q < kKeys / 32; ++q) tmem_wait_ld_x32(s + q * 32);
+                for (int q = 0; q < kHalf / 16; ++q) tmem_wait_ld_x16(s + q * 16);
                 if (C::kSepP) {
                     // S may be overwritten by the next Q K^T from here on
                     tc_fence_before_sync();
@@ -465,60 +489,89 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
                 }
                 FP8ATTN_STAMP(t * 8 + 1, j);
-                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys);
-                if (valid < kKeys) {
+                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys) - h * kHalf;
+                if (valid < kHalf) {
 #pragma unroll
-                    for (int i = 0; i < kKeys; ++i)
+                    for (int i = 0; i < kHalf; ++i)
                         if (i >= valid) s[i] = kNegInf;
                 }
-                // ---- row maximum of the raw scores ----
+                // ---- row maximum: own half, then the partner's through shared memory ----
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < kKeys; i += 8) {
+                for (int i = 0; i < kHalf; i += 8) {
                     mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
                     mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
                     mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
                     mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
                 }
-                const float m_new = max3(m, fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                const float own = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                xchg[j & 1][t][h][row_in_tile] = own;
+                FP8ATTN_STAMP(t * 8 + 5, j);
+                named_barrier_sync(pair_barrier, 64);
+                FP8ATTN_STAMP(t * 8 + 6, j);
+                const float m_tile = fmaxf(own, xchg[j & 1][t][h ^ 1][row_in_tile]);
+                // Lazy reference update: a row keeps its reference m while the new scores
+                // stay within kSlack (log2 units) above it, so its P values reach at most
+                // 2^(lift + kSlack) -- 430 < 448 for e4m3 -- and O needs no rescale.
+                const bool moved = (m_tile - m) * c > kSlack;     // true on the first step (m = -inf)
                 // P V of the previous step must be done before O is rescaled or P rewritten
                 bool pv_done = !(C::kSepP && j > 0);
-                if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
+                if (j == 0) {
+                    m = m_tile;
+                } else if (__any_sync(0xffffffffu, moved)) {
+                    FP8ATTN_STAMP(t * 8 + 7, j);
                     if (!pv_done) {
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                         pv_done = true;
                     }
-                    // the running maximum moved for some row of this warp: rescale O and l
+                    // the reference moved for some row of this warp: rescale O and l
+                    const float m_new = moved ? m_tile : m;
                     const float f = ex2((m - m_new) * c);
+                    m = m_new;
                     const uint64_t ff = pack2(f, f);
                     l2a = mul2(l2a, ff);
                     l2b = mul2(l2b, ff);
 #pragma unroll
-                    for (int q = 0; q < kD / 32; ++q) {
-                        uint32_t o[32];
-                        tmem_ld_x32(tO + q * 32, o);
-                        tmem_wait_ld_x32(o);
+                    for (int q = 0; q < kOHalf / 16; ++q) {
+                        uint32_t o[16];
+                        tmem_ld_x16(tO + q * 16, o);
+                        tmem_wait_ld_x16(o);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                        tmem_st_x32(tO + q * 32, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st_x16(tO + q * 16, o);
                     }
                 }
-                m = m_new;
                 const float nb = lift - m * c;
                 const uint64_t nbnb = pack2(nb, nb);
                 FP8ATTN_STAMP(t * 8 + 2, j);
                 // ---- p = 2^(c*s - c*m + lift), row sums, P tile into tensor memory ----
 #pragma unroll
-                for (int q = 0; q < kKeys / 32; ++q) {
-                    uint32_t p[kFp8 ? 8 : 16];
+                for (int q = 0; q < kHalf / 16; ++q) {
+                    uint32_t p[kFp8 ? 4 : 8];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const uint32_t* cur = s + q * 32 + i;
-                        float x0, x1, x2, x3;
-                        unpack2(fma2(pack2(__uint_as_float(cur[0]), __uint_as_float(cur[1])), cc, nbnb), x0, x1);
-                        unpack2(fma2(pack2(__uint_as_float(cur[2]), __uint_as_float(cur[3])), cc, nbnb), x2, x3);
-                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                    for (int i = 0; i < 16; i += 4) {
+                        const uint32_t* cur = s + q * 16 + i;
+                        const uint64_t xa = fma2(pack2(__uint_as_float(cur[0]), __uint_as_float(cur[1])), cc, nbnb);
+                        const uint64_t xb = fma2(pack2(__uint_as_float(cur[2]), __uint_as_float(cur[3])), cc, nbnb);
+                        float p0, p1, p2, p3;
+                        {
+                            float x0, x1;
+                            unpack2(xa, x0, x1);
+                            p0 = ex2(x0);
+                            p1 = ex2(x1);
+                        }
+                        if (kPolyEvery > 0 && ((i / 4) % kPolyEvery) == kPolyEvery - 1) {
+                            // this pair goes to the FMA pipe to take load off the MUFU
+                            float x2, x3;
+                            unpack2(xb, x2, x3);
+                            exp2_poly2<!kFp8>(pack2(fmaxf(x2, -120.f), fmaxf(x3, -120.f)), p2, p3);
+                        } else {
+                            float x2, x3;
+                            unpack2(xb, x2, x3);
+                            p2 = ex2(x2);
+                            p3 = ex2(x3);
+                        }
                         l2a = add2(l2a, pack2(p0, p1));
                         l2b = add2(l2b, pack2(p2, p3));
                         if (kFp8) {
@@ -532,8 +585,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                     }
-                    if (kFp8) tmem_st_x8(tP + q * 8, p);
-                    else tmem_st_x16(tP + q * 16, p);
+                    if (kFp8) tmem_st_x4(tP + q * 4, p);
+                    else tmem_st_x8(tP + q * 8, p);
                 }
                 FP8ATTN_STAMP(t * 8 + 3, j);
                 tmem_wait_st();
@@ -542,22 +595,26 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
                 FP8ATTN_STAMP(t * 8 + 4, j);
             }
+            // ---- row sum: this half plus the partner's ----
             float l;
             {
                 float a0, a1, b0, b1;
                 unpack2(l2a, a0, a1);
                 unpack2(l2b, b0, b1);
-                l = (a0 + a1) + (b0 + b1);
+                const float own = (a0 + a1) + (b0 + b1);
+                xchg[nkv & 1][t][h][row_in_tile] = own;
+                named_barrier_sync(pair_barrier, 64);
+                l = own + xchg[nkv & 1][t][h ^ 1][row_in_tile];
             }
-            // ---- epilogue: out = s_v * O / l ----
+            // ---- epilogue: out = s_v * O / l, this thread's half of the columns ----
             w.wait(smem_u32(&bars.o_full[t]), 0, kWaitOFull);
             tc_fence_after_sync();
             const int64_t row = row0 + t * kTileM + row_in_tile;
             const float inv = sv_scale / l;
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
-                                 ((int64_t)bh * q_rows + row) * kD;
+                                 ((int64_t)bh * q_rows + row) * kD + h * kOHalf;
 #pragma unroll
-            for (int q = 0; q < kD / 32; ++q) {
+            for (int q = 0; q < kOHalf / 32; ++q) {
                 uint32_t o[32];
                 tmem_ld_x32(tO + q * 32, o);
                 tmem_wait_ld_x32(o);
