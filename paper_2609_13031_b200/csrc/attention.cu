@@ -37,16 +37,23 @@ constexpr int kTileM = 128;           // query rows per tile
 #ifndef FP8ATTN_POLY_EVERY
 #define FP8ATTN_POLY_EVERY 2
 #endif
-constexpr int kSoftmaxWarps = 16;
-constexpr int kQkWarp = 16, kTmaWarp = 17, kPvWarp0 = 18;   // warps 18, 19: P V of tile 0, 1
-constexpr int kNumThreads = 640;      // 16 softmax warps + MMA warp + TMA warp + 2 spare
+#ifndef FP8ATTN_SPLIT
+#define FP8ATTN_SPLIT 1
+#endif
+// kSplit threads share a query row, each owning 1/kSplit of the key columns of a step.
+constexpr int kSplit = FP8ATTN_SPLIT;
+static_assert(kSplit == 1 || kSplit == 2, "row split");
+constexpr int kSoftmaxWarps = 8 * kSplit;
+constexpr int kQkWarp = kSoftmaxWarps, kTmaWarp = kSoftmaxWarps + 1, kPvWarp0 = kSoftmaxWarps + 2;
+constexpr int kNumThreads = (kSoftmaxWarps + 4) * 32;
 // Register budgets after setmaxnreg.  The CTA's register pool is what it was
-// launched with (640 threads x 96); setmaxnreg.inc waits in hardware until the pool
-// can serve it, so the budgets must fit: 16*32*104 + 4*32*56 = 60416 <= 61440.
-constexpr int kRegsSoftmax = 104;
+// launched with (threads x launch registers); setmaxnreg.inc waits in hardware
+// until the pool can serve it, so the budgets must fit in it.
+constexpr int kLaunchRegs = kSplit == 2 ? 96 : 168;
+constexpr int kRegsSoftmax = kSplit == 2 ? 104 : 224;
 constexpr int kRegsOther = 56;
-static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + (kNumThreads - kSoftmaxWarps * 32) * kRegsOther <=
-                  kNumThreads * 96, "setmaxnreg budgets exceed the CTA's register pool");
+static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kNumThreads * kLaunchRegs,
+              "setmaxnreg budgets exceed the CTA's register pool");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
@@ -100,13 +107,19 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 struct Waiter {
     uint32_t* status;
     bool dead;
+    // kBackoffNs > 0: sleep that long between polls.  For waits with plenty of slack
+    // (the TMA producer runs several stages ahead) this keeps the polling out of
+    // the instruction queue that the softmax warps' MUFU and barrier traffic uses.
+    template <uint32_t kBackoffNs = 0>
     __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, uint32_t what) {
         if (dead) return false;
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_test_wait(bar, parity)) return true;
         uint64_t t0 = globaltimer_ns();
         for (;;) {
-            for (int i = 0; i < 64; ++i)
+            for (int i = 0; i < 64; ++i) {
                 if (mbar_try_wait(bar, parity)) return true;
+                if (kBackoffNs > 0) __nanosleep(kBackoffNs);
+            }
             // another CTA already gave up: do not wait out the limit here as well
             if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { dead = true; return false; }
             if (globaltimer_ns() - t0 > kWaitLimitNs) break;
@@ -209,6 +222,9 @@ __device__ __forceinline__ void tmem_wait_ld_x16(uint32_t* r) {
                  :
                  : "memory");
 }
+__device__ __forceinline__ void named_barrier_arrive(uint32_t id, uint32_t threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -239,13 +255,43 @@ __device__ long long* g_trace_buf;
 #define FP8ATTN_TRACE_INIT() long long* const trace_buf = (blockIdx.x == 0) ? g_trace_buf : nullptr
 #define FP8ATTN_STAMP(slot, j)                                                         \
     do {                                                                               \
-        if (trace_buf != nullptr && lane == 0 && (warp >= 16 || (warp & 7) == 0) && (j) >= 64 && (j) < 80)                \
+        if (trace_buf != nullptr && lane == 0 && (warp >= kSoftmaxWarps || (warp % (4 * kSplit)) == 0) && (j) >= 64 && (j) < 80)                \
             trace_buf[((j) - 64) * 32 + (slot)] = clock64();                           \
     } while (0)
 #else
 #define FP8ATTN_TRACE_INIT() do { } while (0)
 #define FP8ATTN_STAMP(slot, j) do { } while (0)
 #endif
+
+// tcgen05.ld / wait / st of kCols consecutive columns (multiple of 16) in as few
+// instructions as possible
+template <int kCols>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t* r) {
+#pragma unroll
+    for (int q = 0; q + 32 <= kCols; q += 32) tmem_ld_x32(taddr + q, r + q);
+    if (kCols % 32) tmem_ld_x16(taddr + (kCols / 32) * 32, r + (kCols / 32) * 32);
+}
+template <int kCols>
+__device__ __forceinline__ void tmem_wait_ld_cols(uint32_t* r) {
+#pragma unroll
+    for (int q = 0; q + 32 <= kCols; q += 32) tmem_wait_ld_x32(r + q);
+    if (kCols % 32) tmem_wait_ld_x16(r + (kCols / 32) * 32);
+}
+template <int kCols>
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) {
+    static_assert(kCols == 4 || kCols == 8 || kCols == 16 || kCols == 32, "store width");
+    if (kCols == 4) tmem_st_x4(taddr, r);
+    else if (kCols == 8) tmem_st_x8(taddr, r);
+    else if (kCols == 16) tmem_st_x16(taddr, r);
+    else tmem_st_x32(taddr, r);
+}
+
+// Named barriers (hardware-blocking, no polling).  1..8: the two warps sharing
+// rows when a row is split; 9, 10: whose turn the exponential phase is;
+// 11 + t: "S_t is in registers" (softmax -> Q K^T issuer); 13 + t: "P_t is in
+// tensor memory" (softmax -> P V issuer of tile t).
+constexpr uint32_t kTurnBarrier0 = 9, kSFreeBarrier0 = 11, kPFullBarrier0 = 13;
+constexpr uint32_t kSignalThreads = 128 * kSplit + 32;   // one tile's softmax threads + the issuer warp
 
 struct KernelArgs {
     const float* scale_q; const float* scale_k; const float* scale_v;
@@ -302,8 +348,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.s_free[t]), 8);
-            mbar_init(smem_u32(&bars.p_full[t]), 8);
+            mbar_init(smem_u32(&bars.s_free[t]), 4 * kSplit);
+            mbar_init(smem_u32(&bars.p_full[t]), 4 * kSplit);
             mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
         }
@@ -340,14 +386,14 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         for (int j = 0; j < nkv; ++j) {
             const int s = j % C::kStages;
             const uint32_t ph = (j / C::kStages) & 1;
-            w.wait(smem_u32(&bars.k_empty[s]), ph ^ 1, kWaitKEmpty);
+            w.wait<400>(smem_u32(&bars.k_empty[s]), ph ^ 1, kWaitKEmpty);
             if (elect_one()) {
                 mbar_arrive_expect_tx(smem_u32(&bars.k_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
                     tma_load_3d(sK + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_k,
                                 b * C::kBoxCols, j * kKeys, bh, smem_u32(&bars.k_full[s]));
             }
-            w.wait(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
+            w.wait<400>(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
             if (elect_one()) {
                 mbar_arrive_expect_tx(smem_u32(&bars.v_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
@@ -403,7 +449,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             for (int t = 0; t < ntiles; ++t) {
                 // S_t is free once its rows sit in registers; where P is written over S,
                 // only once P V of this step has consumed it
-                if (C::kSepP) w.wait(smem_u32(&bars.s_free[t]), j & 1, kWaitSFree);
+                if (C::kSepP) named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
                 else w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
                 tc_fence_after_sync();
                 FP8ATTN_STAMP(20 + t, j);
@@ -423,7 +469,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             for (int j = 0; j < nkv; ++j) {
                 const int sv = j % C::kStages;
                 w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
-                w.wait(smem_u32(&bars.p_full[t]), j & 1, kWaitPFull);
+                named_barrier_sync(kPFullBarrier0 + t, kSignalThreads);
                 tc_fence_after_sync();
                 FP8ATTN_STAMP(16 + t * 2, j);
                 if (elect_one()) {
@@ -444,18 +490,18 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     } else {
         // ========================= softmax + epilogue =========================
         setmaxnreg_inc<kRegsSoftmax>();
-        constexpr int kHalf = kKeys / 2;         // key columns of a step owned by one thread
-        constexpr int kPHalf = C::kPCols / 2;    // P columns owned by one thread
-        constexpr int kOHalf = kD / 2;           // output columns owned by one thread
-        const int t = warp >> 3;                 // query tile
-        const int h = (warp >> 2) & 1;           // column half
+        constexpr int kCols = kKeys / kSplit;          // key columns of a step owned by one thread
+        constexpr int kPColsT = C::kPCols / kSplit;    // P columns owned by one thread
+        constexpr int kOCols = kD / kSplit;            // output columns owned by one thread
+        const int t = warp / (4 * kSplit);             // query tile
+        const int h = (warp >> 2) % kSplit;            // which part of the columns
         if (t < ntiles) {
             const int row_in_tile = (warp & 3) * 32 + lane;
-            const uint32_t pair_barrier = 1 + t * 4 + (warp & 3);   // the two warps that share rows
+            const uint32_t pair_barrier = 1 + t * 4 + (warp & 3);   // the warps that share rows
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0) + h * kHalf;
-            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0) + h * kPHalf;
-            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD + h * kOHalf;
+            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0) + h * kCols;
+            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0) + h * kPColsT;
+            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD + h * kOCols;
             float c = (args.softmax_scale > 0.f ? args.softmax_scale : rsqrtf((float)kD)) *
                       1.4426950408889634f;
             float sv_scale = 1.0f;
@@ -467,73 +513,73 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             // every kPolyEvery-th group of four columns computes two of its exponentials
             // with the polynomial (0 = never): 1 -> 50 %, 2 -> 25 %, 4 -> 12.5 % of all
             constexpr int kPolyEvery = FP8ATTN_POLY_EVERY;
-            constexpr float kSlack = 0.0f;   // exact running maximum: the row maximum maps to 2^lift
             const uint64_t cc = pack2(c, c);
             float m = -INFINITY;
-            uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // partial row sums of this half
+            uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // partial row sums
             constexpr uint32_t kNegInf = 0xff800000u;
+            // The two query tiles take turns on the exponential phase (tile 0 of step j,
+            // tile 1 of step j, tile 0 of step j+1, ...): one tile's MUFU work then runs
+            // under the other's tensor-memory loads, maximum and barrier traffic instead
+            // of both queueing on the MUFU at once and leaving it idle together.
+            const bool ping_pong = ntiles == 2;
+            constexpr uint32_t kTurnThreads = 2 * 128 * kSplit;
+            if (ping_pong && t == 1) named_barrier_arrive(kTurnBarrier0, kTurnThreads);
             for (int j = 0; j < nkv; ++j) {
                 w.wait(smem_u32(&bars.s_full[t]), j & 1, kWaitSFull);
                 tc_fence_after_sync();
                 FP8ATTN_STAMP(t * 8 + 0, j);
-                // ---- this thread's half of the score row into registers ----
-                uint32_t s[kHalf];
-#pragma unroll
-                for (int q = 0; q < kHalf / 16; ++q) tmem_ld_x16(tS + q * 16, s + q * 16);
-#pragma unroll
-                for (int q = 0; q < kHalf / 16; ++q) tmem_wait_ld_x16(s + q * 16);
-                if (C::kSepP) {
+                // ---- this thread's part of the score row into registers ----
+                uint32_t s[kCols];
+                tmem_ld_cols<kCols>(tS, s);
+                tmem_wait_ld_cols<kCols>(s);
+                if (C::kSepP && j + 1 < nkv) {
                     // S may be overwritten by the next Q K^T from here on
                     tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
+                    named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
                 }
                 FP8ATTN_STAMP(t * 8 + 1, j);
-                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys) - h * kHalf;
-                if (valid < kHalf) {
+                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys) - h * kCols;
+                if (valid < kCols) {
 #pragma unroll
-                    for (int i = 0; i < kHalf; ++i)
+                    for (int i = 0; i < kCols; ++i)
                         if (i >= valid) s[i] = kNegInf;
                 }
-                // ---- row maximum: own half, then the partner's through shared memory ----
+                // ---- row maximum (own columns, then the partner's through shared memory) ----
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < kHalf; i += 8) {
+                for (int i = 0; i < kCols; i += 8) {
                     mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
                     mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
                     mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
                     mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
                 }
-                const float own = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                xchg[j & 1][t][h][row_in_tile] = own;
-                FP8ATTN_STAMP(t * 8 + 5, j);
-                named_barrier_sync(pair_barrier, 64);
-                FP8ATTN_STAMP(t * 8 + 6, j);
-                const float m_tile = fmaxf(own, xchg[j & 1][t][h ^ 1][row_in_tile]);
-                // Lazy reference update: a row keeps its reference m while the new scores
-                // stay within kSlack (log2 units) above it, so its P values reach at most
-                // 2^(lift + kSlack) -- 430 < 448 for e4m3 -- and O needs no rescale.
-                const bool moved = (m_tile - m) * c > kSlack;     // true on the first step (m = -inf)
+                float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                if (kSplit == 2) {
+                    xchg[j & 1][t][h][row_in_tile] = m_tile;
+                    FP8ATTN_STAMP(t * 8 + 5, j);
+                    named_barrier_sync(pair_barrier, 64);
+                    FP8ATTN_STAMP(t * 8 + 6, j);
+                    m_tile = fmaxf(m_tile, xchg[j & 1][t][h ^ 1][row_in_tile]);
+                }
+                // The reference maximum is the exact running maximum: the row maximum of
+                // the keys seen so far maps to 2^lift.
+                const float m_new = fmaxf(m, m_tile);
                 // P V of the previous step must be done before O is rescaled or P rewritten
                 bool pv_done = !(C::kSepP && j > 0);
-                if (j == 0) {
-                    m = m_tile;
-                } else if (__any_sync(0xffffffffu, moved)) {
+                if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
                     FP8ATTN_STAMP(t * 8 + 7, j);
                     if (!pv_done) {
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                         pv_done = true;
                     }
-                    // the reference moved for some row of this warp: rescale O and l
-                    const float m_new = moved ? m_tile : m;
+                    // the maximum moved for some row of this warp: rescale O and l
                     const float f = ex2((m - m_new) * c);
-                    m = m_new;
                     const uint64_t ff = pack2(f, f);
                     l2a = mul2(l2a, ff);
                     l2b = mul2(l2b, ff);
 #pragma unroll
-                    for (int q = 0; q < kOHalf / 16; ++q) {
+                    for (int q = 0; q < kOCols / 16; ++q) {
                         uint32_t o[16];
                         tmem_ld_x16(tO + q * 16, o);
                         tmem_wait_ld_x16(o);
@@ -542,33 +588,33 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         tmem_st_x16(tO + q * 16, o);
                     }
                 }
+                m = m_new;
                 const float nb = lift - m * c;
                 const uint64_t nbnb = pack2(nb, nb);
+                if (ping_pong) named_barrier_sync(kTurnBarrier0 + t, kTurnThreads);
                 FP8ATTN_STAMP(t * 8 + 2, j);
                 // ---- p = 2^(c*s - c*m + lift), row sums, P tile into tensor memory ----
+                // chunks of 32 keys (a last one of 16 where the column count asks for it)
 #pragma unroll
-                for (int q = 0; q < kHalf / 16; ++q) {
-                    uint32_t p[kFp8 ? 4 : 8];
+                for (int k0 = 0; k0 < kCols; k0 += 32) {
+                    constexpr int kPPer32 = kFp8 ? 8 : 16;
+                    uint32_t p[kPPer32];
+                    const int n = (kCols - k0) < 32 ? (kCols - k0) : 32;
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const uint32_t* cur = s + q * 16 + i;
+                    for (int i = 0; i < 32; i += 4) {
+                        if (i >= n) break;
+                        const uint32_t* cur = s + k0 + i;
                         const uint64_t xa = fma2(pack2(__uint_as_float(cur[0]), __uint_as_float(cur[1])), cc, nbnb);
                         const uint64_t xb = fma2(pack2(__uint_as_float(cur[2]), __uint_as_float(cur[3])), cc, nbnb);
-                        float p0, p1, p2, p3;
-                        {
-                            float x0, x1;
-                            unpack2(xa, x0, x1);
-                            p0 = ex2(x0);
-                            p1 = ex2(x1);
-                        }
+                        float p0, p1, p2, p3, x0, x1, x2, x3;
+                        unpack2(xa, x0, x1);
+                        unpack2(xb, x2, x3);
+                        p0 = ex2(x0);
+                        p1 = ex2(x1);
                         if (kPolyEvery > 0 && ((i / 4) % kPolyEvery) == kPolyEvery - 1) {
                             // this pair goes to the FMA pipe to take load off the MUFU
-                            float x2, x3;
-                            unpack2(xb, x2, x3);
                             exp2_poly2<!kFp8>(pack2(fmaxf(x2, -120.f), fmaxf(x3, -120.f)), p2, p3);
                         } else {
-                            float x2, x3;
-                            unpack2(xb, x2, x3);
                             p2 = ex2(x2);
                             p3 = ex2(x3);
                         }
@@ -581,40 +627,43 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                             p[i / 2 + 1] = pack_bf16x2(p2, p3);
                         }
                     }
-                    if (q == 0 && !pv_done) {
+                    if (k0 == 0 && !pv_done) {
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                     }
-                    if (kFp8) tmem_st_x4(tP + q * 4, p);
-                    else tmem_st_x8(tP + q * 8, p);
+                    if (n == 32) tmem_st_cols<kPPer32>(tP + (k0 / 32) * kPPer32, p);
+                    else tmem_st_cols<kPPer32 / 2>(tP + (k0 / 32) * kPPer32, p);
                 }
+                if (ping_pong) named_barrier_arrive(kTurnBarrier0 + (t ^ 1), kTurnThreads);
                 FP8ATTN_STAMP(t * 8 + 3, j);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
+                named_barrier_arrive(kPFullBarrier0 + t, kSignalThreads);
                 FP8ATTN_STAMP(t * 8 + 4, j);
             }
-            // ---- row sum: this half plus the partner's ----
+            if (ping_pong && t == 0) named_barrier_sync(kTurnBarrier0, kTurnThreads);   // last turn token
+            // ---- row sum (plus the partner's) ----
             float l;
             {
                 float a0, a1, b0, b1;
                 unpack2(l2a, a0, a1);
                 unpack2(l2b, b0, b1);
-                const float own = (a0 + a1) + (b0 + b1);
-                xchg[nkv & 1][t][h][row_in_tile] = own;
-                named_barrier_sync(pair_barrier, 64);
-                l = own + xchg[nkv & 1][t][h ^ 1][row_in_tile];
+                l = (a0 + a1) + (b0 + b1);
+                if (kSplit == 2) {
+                    xchg[nkv & 1][t][h][row_in_tile] = l;
+                    named_barrier_sync(pair_barrier, 64);
+                    l += xchg[nkv & 1][t][h ^ 1][row_in_tile];
+                }
             }
-            // ---- epilogue: out = s_v * O / l, this thread's half of the columns ----
+            // ---- epilogue: out = s_v * O / l, this thread's share of the columns ----
             w.wait(smem_u32(&bars.o_full[t]), 0, kWaitOFull);
             tc_fence_after_sync();
             const int64_t row = row0 + t * kTileM + row_in_tile;
             const float inv = sv_scale / l;
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
-                                 ((int64_t)bh * q_rows + row) * kD + h * kOHalf;
+                                 ((int64_t)bh * q_rows + row) * kD + h * kOCols;
 #pragma unroll
-            for (int q = 0; q < kOHalf / 32; ++q) {
+            for (int q = 0; q < kOCols / 32; ++q) {
                 uint32_t o[32];
                 tmem_ld_x32(tO + q * 32, o);
                 tmem_wait_ld_x32(o);
