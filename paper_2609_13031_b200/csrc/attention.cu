@@ -37,6 +37,9 @@ constexpr int kTileM = 128;           // query rows per tile
 #ifndef FP8ATTN_POLY_EVERY
 #define FP8ATTN_POLY_EVERY 2
 #endif
+#ifndef FP8ATTN_PINGPONG
+#define FP8ATTN_PINGPONG 0
+#endif
 #ifndef FP8ATTN_SPLIT
 #define FP8ATTN_SPLIT 1
 #endif
@@ -521,7 +524,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             // tile 1 of step j, tile 0 of step j+1, ...): one tile's MUFU work then runs
             // under the other's tensor-memory loads, maximum and barrier traffic instead
             // of both queueing on the MUFU at once and leaving it idle together.
-            const bool ping_pong = ntiles == 2;
+            const bool ping_pong = FP8ATTN_PINGPONG && ntiles == 2;
             constexpr uint32_t kTurnThreads = 2 * 128 * kSplit;
             if (ping_pong && t == 1) named_barrier_arrive(kTurnBarrier0, kTurnThreads);
             for (int j = 0; j < nkv; ++j) {
