@@ -27,6 +27,9 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from an ncu capture of the
+# same workload (summaries under profiles/); None where no capture exists.
+NCU_DRAM_BYTES_PER_LAUNCH = {"C3": 219.7e6 + 138.0e6}
 NOMINAL_FP8_OVER_BF16 = 2.0           # dense tensor peak ratio (4.5 / 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -71,7 +74,7 @@ class ClockSampler(threading.Thread):
     def run(self):
         while not self.stop_flag.is_set():
             self.sample()
-            self.stop_flag.wait(0.2)
+            self.stop_flag.wait(0.1)
 
     def result(self):
         self.stop_flag.set()
@@ -148,7 +151,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -166,7 +169,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2609_13031_b200 import api
+    from paper_2609_13031_b200 import api, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -228,11 +231,7 @@ def main():
         return torch.cuda.Event(enable_timing=True)
 
     def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(ms, "cuda")
 
     # ---- device-resident timing: K steps, events per sub-kernel group ----
     for _ in range(args.warmup):
@@ -335,7 +334,7 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "kernel": "icl_attention_kernel<fp8>",
                          "achieved": tf_attn, "peak": peak_fp8, "unit": "TFLOP/s",
-                         "frac": tf_attn / peak_fp8, "traffic": None,
+                         "frac": tf_attn / peak_fp8, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
                          "peak_source": f"2 x bf16_tflops_sustained ({peak_kind}), nominal fp8:bf16 ratio",
                          "frac_of_burst_peak": tf_attn / peak_fp8_burst,
                          "frac_of_nominal_4500": tf_attn / 4500.0},

@@ -106,6 +106,16 @@ def test_fp8_c3_full_size_sampled():
     check_fp8_case(W.CONFIGS["C3"], n_sample=40, named_config=True)
 
 
+def test_fp8_c4_full_size_sampled():
+    # B=4 independent tables, 262,144 train rows each, keys with mean 3: diffuse softmax
+    check_fp8_case(W.CONFIGS["C4"], n_sample=12, diffuse=True, named_config=True)
+
+
+def test_fp8_c5_full_size_sampled():
+    # 1,048,576 train rows: the large-table regime
+    check_fp8_case(W.CONFIGS["C5"], n_sample=12, named_config=True)
+
+
 def test_fp8_custom_softmax_scale():
     check_fp8_case(W.CONFIGS["C1"].scaled(300, 40), alpha=0.05)
 
@@ -127,6 +137,10 @@ def test_bf16_d128_small():
 
 def test_bf16_c2_sampled():
     check_bf16_case(W.CONFIGS["C2"], n_sample=64)
+
+
+def test_bf16_c3_full_size_sampled():
+    check_bf16_case(W.CONFIGS["C3"], n_sample=24)
 
 
 # ---- structure of the ICL layer -------------------------------------------------------
