@@ -44,7 +44,8 @@ def load_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs
+    (one streaming ``nvidia-smi -lms 100`` child, read line by line)."""
 
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -53,32 +54,33 @@ class ClockSampler(threading.Thread):
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
-        self.index = index
-        self.stop_flag = threading.Event()
         self.sm, self.max_sm, self.reasons = [], 0.0, set()
-
-    def sample(self):
         try:
-            out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                  "--format=csv,noheader,nounits"], capture_output=True, text=True,
-                                 timeout=5).stdout.strip().splitlines()[0]
-            f = [x.strip() for x in out.split(",")]
-            self.sm.append(float(f[0]))
-            self.max_sm = float(f[1])
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def run(self):
+        if self.proc is None:
+            return
+        for line in self.proc.stdout:
+            f = [x.strip() for x in line.split(",")]
+            try:
+                self.sm.append(float(f[0]))
+                self.max_sm = float(f[1])
+            except (ValueError, IndexError):
+                continue
             for name, val in zip(self.NAMES, f[2:]):
                 if val.lower().startswith("active"):
                     self.reasons.add(name)
-        except Exception:
-            pass
-
-    def run(self):
-        while not self.stop_flag.is_set():
-            self.sample()
-            self.stop_flag.wait(0.1)
 
     def result(self):
-        self.stop_flag.set()
-        self.join(timeout=10)
+        if self.proc is not None:
+            self.proc.terminate()          # our own child, by handle
+            self.join(timeout=10)
         if not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
         return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_sm,
@@ -151,7 +153,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -243,6 +245,15 @@ def main():
         raise RuntimeError(f"device status {status}")
     sampler = ClockSampler(local)
     sampler.start()
+    # keep the GPU busy (untimed) until the sampler delivers, so every sample is under load
+    for _ in range(200):
+        quantize_all()
+        attention_fp8()
+        torch.cuda.synchronize()
+        if sampler.sm:
+            break
+    sampler.sm.clear()
+    sampler.reasons.clear()
     launches0 = api.launch_count()
     marks = []
     sync_all()
