@@ -1,16 +1,19 @@
 // Fused ICL attention for sm_100a: train->train and test->train in one launch.
 //
 // One CTA owns up to 256 query rows (two 128-row tiles) of one (b,h) and walks
-// over all train keys in steps of kKeys keys.  Warp roles:
-//   warps 0-7   softmax of query tile 0: two threads per row, each owning half of
-//               the key columns of a step (warps 0-3: first half, 4-7: second half)
-//   warps 8-15  softmax of query tile 1, same split
-//   warp  16    issues the Q K^T tcgen05.mma of both tiles (one elected lane)
-//   warp  17    TMA producer for Q, K and V tiles
-//   warps 18-19 issue the P V tcgen05.mma of tile 0 and tile 1
-// Four softmax warps per scheduler hide each other's tensor-memory, MUFU and
-// barrier latencies; the two threads of a row exchange their partial maxima
-// through shared memory once per step.
+// over all train keys in steps of kKeys keys.  Warp roles (default build):
+//   warps 0-3   softmax of query tile 0, one row per thread
+//   warps 4-7   softmax of query tile 1
+//   warp  8     issues the Q K^T tcgen05.mma of both tiles (one elected lane)
+//   warp  9     TMA producer for Q, K and V tiles
+//   warps 10-11 issue the P V tcgen05.mma of tile 0 and tile 1
+// Q K^T and P V are issued from different warps because a single warp cannot
+// issue tcgen05 instructions of this size fast enough to keep the tensor core fed.
+// Build options (compile-time, for experiments): FP8ATTN_SPLIT=2 lets two threads
+// share a row (16 softmax warps; they exchange partial maxima through shared memory
+// once per step), FP8ATTN_PINGPONG=1 makes the two tiles take strict turns on the
+// exponential phase, FP8ATTN_POLY_EVERY sets the share of exponentials computed by
+// a polynomial on the FMA pipe instead of the MUFU.
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
