@@ -101,6 +101,39 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
                          void* out_train_bf16, void* out_test_bf16,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Variants of the two forward calls with a flags word.
+ *
+ * FP8ATTN_TEST_ROWS_USE_KV_HEAD0: grouped-query test->train attention as in
+ * TabPFN-v3 (paper appendix, noise-experiment details: "test rows attend to the
+ * first K,V head"): the test queries of every head h of a table attend to the
+ * keys and values of head 0 of that table (and use head 0's K and V scales; the
+ * query scale stays head h's train-query scale).  Train rows are unaffected.
+ * K and V are still passed, and were quantized, as full [B,H,n_train,d] tensors,
+ * so both attention calls consume the same quantized K/V entries.
+ * Unknown flag bits return FP8ATTN_ERR_INVALID_ARG.  flags = 0 is the plain call.
+ */
+#define FP8ATTN_TEST_ROWS_USE_KV_HEAD0 1u
+int fp8attn_icl_forward_ex(const void* q_train_fp8, const void* q_test_fp8,
+                           const void* k_fp8, const void* v_fp8,
+                           const float* scale_q, const float* scale_k, const float* scale_v,
+                           int B, int H, int64_t n_train, int64_t n_test, int d,
+                           float softmax_scale, uint32_t flags,
+                           void* out_train_bf16, void* out_test_bf16,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+int bf16attn_icl_forward_ex(const void* q_train, const void* q_test, const void* k, const void* v,
+                            int B, int H, int64_t n_train, int64_t n_test, int d,
+                            float softmax_scale, uint32_t flags,
+                            void* out_train_bf16, void* out_test_bf16,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The paper's dispatch gate (Method section: the quantization overhead is
+ * amortised for N > 8192 train rows, and the final configuration uses FP8 only
+ * then).  Host-only helper, returns 1 if the FP8 path should be used for this
+ * many train rows, else 0 (use bf16attn_icl_forward).  Policy, not enforced:
+ * fp8attn_icl_forward itself runs at any size. */
+#define FP8ATTN_GATE_TRAIN_ROWS 8192
+int fp8attn_gate_use_fp8(int64_t n_train);
+
 /* Allocation-free quantizer (the paper has no counterpart; this is a
  * packaging variant of fp8attn_quantize, same arithmetic, same results).
  *

@@ -22,7 +22,10 @@ EXPORTS = (
     "fp8attn_quantize", "fp8attn_icl_forward", "bf16attn_icl_forward",
     "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
+    "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
 )
+TEST_ROWS_USE_KV_HEAD0 = 1
+GATE_TRAIN_ROWS = 8192
 
 _lib = None
 
@@ -53,6 +56,15 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_icl_forward.restype = i32
     lib.fp8attn_icl_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i64, i32, f32,
                                         vp, vp, vp, sz, vp]
+    u32 = ctypes.c_uint32
+    lib.fp8attn_icl_forward_ex.restype = i32
+    lib.fp8attn_icl_forward_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, u32,
+                                           vp, vp, vp, sz, vp]
+    lib.bf16attn_icl_forward_ex.restype = i32
+    lib.bf16attn_icl_forward_ex.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, u32, vp, vp,
+                                            vp, sz, vp]
+    lib.fp8attn_gate_use_fp8.restype = i32
+    lib.fp8attn_gate_use_fp8.argtypes = [i64]
     lib.bf16attn_icl_forward.restype = i32
     lib.bf16attn_icl_forward.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, vp, vp, vp,
                                          sz, vp]
@@ -136,9 +148,15 @@ def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor
     return out, scale_out
 
 
+def gate_use_fp8(n_train: int) -> bool:
+    """fp8attn_gate_use_fp8: the paper's N > 8192 dispatch rule."""
+    return bool(load().fp8attn_gate_use_fp8(int(n_train)))
+
+
 def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
-                    softmax_scale: float = 0.0, out_train=None, out_test=None):
-    """fp8attn_icl_forward on uint8 e4m3 tensors; returns (out_train, out_test) bf16."""
+                    softmax_scale: float = 0.0, out_train=None, out_test=None, flags: int = 0):
+    """fp8attn_icl_forward (flags == 0) / fp8attn_icl_forward_ex on uint8 e4m3
+    tensors; returns (out_train, out_test) bf16."""
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
     for t in (q_train, k, v):
@@ -147,6 +165,14 @@ def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
         out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
     if out_test is None and n_test > 0:
         out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+    if flags:
+        rc = load().fp8attn_icl_forward_ex(
+            _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v),
+            _ptr(scale_q), _ptr(scale_k), _ptr(scale_v), B, H, n_train, n_test, d,
+            float(softmax_scale), int(flags), _ptr(out_train), _ptr(out_test) if n_test else None,
+            _ptr(workspace), workspace.numel(), _stream())
+        _check("fp8attn_icl_forward_ex", rc)
+        return out_train, out_test
     rc = load().fp8attn_icl_forward(
         _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v),
         _ptr(scale_q), _ptr(scale_k), _ptr(scale_v), B, H, n_train, n_test, d,
@@ -157,7 +183,7 @@ def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
 
 
 def icl_forward_bf16(q_train, q_test, k, v, workspace, softmax_scale: float = 0.0,
-                     out_train=None, out_test=None):
+                     out_train=None, out_test=None, flags: int = 0):
     """bf16attn_icl_forward on bf16 tensors; returns (out_train, out_test) bf16."""
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
@@ -167,6 +193,13 @@ def icl_forward_bf16(q_train, q_test, k, v, workspace, softmax_scale: float = 0.
         out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
     if out_test is None and n_test > 0:
         out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+    if flags:
+        rc = load().bf16attn_icl_forward_ex(
+            _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v), B, H, n_train, n_test,
+            d, float(softmax_scale), int(flags), _ptr(out_train), _ptr(out_test) if n_test else None,
+            _ptr(workspace), workspace.numel(), _stream())
+        _check("bf16attn_icl_forward_ex", rc)
+        return out_train, out_test
     rc = load().bf16attn_icl_forward(
         _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v), B, H, n_train, n_test, d,
         float(softmax_scale), _ptr(out_train), _ptr(out_test) if n_test else None,

@@ -36,7 +36,7 @@ int check_device() {
 int forward(bool fp8, const void* q_train, const void* q_test, const void* k, const void* v,
             const float* sq, const float* sk, const float* sv, int B, int H, int64_t n_train,
             int64_t n_test, int d, float softmax_scale, void* out_train, void* out_test,
-            void* workspace, size_t workspace_bytes_, void* stream) {
+            void* workspace, size_t workspace_bytes_, void* stream, uint32_t flags = 0) {
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0 || n_train > 0x7fffff00ll || n_test > 0x7fffff00ll)
@@ -48,6 +48,7 @@ int forward(bool fp8, const void* q_train, const void* q_test, const void* k, co
         (n_test > 0 && (!aligned(q_test, 16) || !aligned(out_test, 16))))
         return FP8ATTN_ERR_INVALID_ARG;
     if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return FP8ATTN_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)FP8ATTN_TEST_ROWS_USE_KV_HEAD0) return FP8ATTN_ERR_INVALID_ARG;
     rc = check_workspace(workspace, workspace_bytes_, B, H);
     if (rc != FP8ATTN_OK) return rc;
     rc = check_device();
@@ -57,6 +58,7 @@ int forward(bool fp8, const void* q_train, const void* q_test, const void* k, co
     p.scale_q = sq; p.scale_k = sk; p.scale_v = sv;
     p.B = B; p.H = H; p.n_train = n_train; p.n_test = n_test; p.d = d;
     p.softmax_scale = softmax_scale;
+    p.flags = flags;
     p.out_train = out_train; p.out_test = out_test;
     p.status = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsStatusOffset);
     return launch_icl_attention(p, fp8, static_cast<cudaStream_t>(stream));
@@ -105,6 +107,28 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
     return forward(false, q_train, q_test, k, v, nullptr, nullptr, nullptr, B, H, n_train, n_test, d,
                    softmax_scale, out_train_bf16, out_test_bf16, workspace, workspace_bytes_, cuda_stream);
 }
+
+int fp8attn_icl_forward_ex(const void* q_train_fp8, const void* q_test_fp8, const void* k_fp8,
+                           const void* v_fp8, const float* scale_q, const float* scale_k,
+                           const float* scale_v, int B, int H, int64_t n_train, int64_t n_test, int d,
+                           float softmax_scale, uint32_t flags, void* out_train_bf16,
+                           void* out_test_bf16, void* workspace, size_t workspace_bytes_,
+                           void* cuda_stream) {
+    return forward(true, q_train_fp8, q_test_fp8, k_fp8, v_fp8, scale_q, scale_k, scale_v, B, H, n_train,
+                   n_test, d, softmax_scale, out_train_bf16, out_test_bf16, workspace, workspace_bytes_,
+                   cuda_stream, flags);
+}
+
+int bf16attn_icl_forward_ex(const void* q_train, const void* q_test, const void* k, const void* v, int B,
+                            int H, int64_t n_train, int64_t n_test, int d, float softmax_scale,
+                            uint32_t flags, void* out_train_bf16, void* out_test_bf16, void* workspace,
+                            size_t workspace_bytes_, void* cuda_stream) {
+    return forward(false, q_train, q_test, k, v, nullptr, nullptr, nullptr, B, H, n_train, n_test, d,
+                   softmax_scale, out_train_bf16, out_test_bf16, workspace, workspace_bytes_, cuda_stream,
+                   flags);
+}
+
+int fp8attn_gate_use_fp8(int64_t n_train) { return n_train > FP8ATTN_GATE_TRAIN_ROWS ? 1 : 0; }
 
 size_t fp8attn_workspace_bytes(int B, int H, int64_t, int64_t, int) {
     if (B <= 0 || H <= 0) return 0;

@@ -304,6 +304,8 @@ struct KernelArgs {
     void* out_train; void* out_test;
     int64_t n_train, n_test;
     int blocks_train, blocks_test;   // 256-row query blocks per head
+    int heads;                       // H, to find head 0 of a table
+    int test_kv_head0;               // test rows read K, V and their scales from head 0 of their table
     float softmax_scale;
     uint32_t* status;
 };
@@ -338,6 +340,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     const int64_t n_keys = args.n_train;
     const int nkv = (int)((n_keys + kKeys - 1) / kKeys);
     const CUtensorMap* map_q = is_test ? &map_q_test : &map_q_train;
+    // grouped-query variant: every test query head attends to the first K/V head of its table
+    const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
 
     // A device error recorded earlier (and not yet read back by the host) is sticky:
     // nothing runs until fp8attn_last_device_status() has cleared it.
@@ -397,14 +401,14 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 mbar_arrive_expect_tx(smem_u32(&bars.k_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
                     tma_load_3d(sK + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_k,
-                                b * C::kBoxCols, j * kKeys, bh, smem_u32(&bars.k_full[s]));
+                                b * C::kBoxCols, j * kKeys, bh_kv, smem_u32(&bars.k_full[s]));
             }
             w.wait<400>(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
             if (elect_one()) {
                 mbar_arrive_expect_tx(smem_u32(&bars.v_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
                     tma_load_3d(sV + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_v,
-                                b * C::kBoxCols, j * kKeys, bh, smem_u32(&bars.v_full[s]));
+                                b * C::kBoxCols, j * kKeys, bh_kv, smem_u32(&bars.v_full[s]));
             }
             __syncwarp();
         }
@@ -512,8 +516,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                       1.4426950408889634f;
             float sv_scale = 1.0f;
             if (kFp8) {
-                c *= args.scale_q[bh] * args.scale_k[bh];
-                sv_scale = args.scale_v[bh];
+                c *= args.scale_q[bh] * args.scale_k[bh_kv];
+                sv_scale = args.scale_v[bh_kv];
             }
             const float lift = kFp8 ? 8.0f : 0.0f;
             // every kPolyEvery-th group of four columns computes two of its exponentials
@@ -715,6 +719,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     a.blocks_train = (int)((p.n_train + 2 * kTileM - 1) / (2 * kTileM));
     a.blocks_test = (int)((p.n_test + 2 * kTileM - 1) / (2 * kTileM));
     a.softmax_scale = p.softmax_scale;
+    a.heads = p.H;
+    a.test_kv_head0 = (p.flags & FP8ATTN_TEST_ROWS_USE_KV_HEAD0) ? 1 : 0;
     a.status = p.status;
     const int64_t grid = heads * (a.blocks_train + a.blocks_test);
     if (grid > 0x7fffffffll) return FP8ATTN_ERR_UNSUPPORTED;

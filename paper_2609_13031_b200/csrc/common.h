@@ -35,6 +35,7 @@ struct AttnParams {
     const float* scale_q; const float* scale_k; const float* scale_v;  // NULL for bf16
     int B, H; int64_t n_train, n_test; int d;
     float softmax_scale;
+    uint32_t flags;    // FP8ATTN_* forward flags
     void* out_train; void* out_test;
     uint32_t* status;  // workspace status words
 };

@@ -38,3 +38,13 @@ def test_host_only_entry_points():
     assert api.workspace_bytes(1, 8) >= 256 + 32
     assert api.workspace_bytes(4, 4) % 256 == 0
     assert api.workspace_bytes(0, 4) == 0
+
+
+def test_dispatch_gate_matches_the_paper_constant():
+    import os
+    from helpers import read_golden_table
+    gold = dict(read_golden_table(os.path.join(ROOT, "tests", "golden", "paper_constants.txt")))
+    gate = int(float(gold["fp8_gate_train_rows"]))          # Method section: N > 8192
+    assert api.GATE_TRAIN_ROWS == gate
+    assert not api.gate_use_fp8(gate) and api.gate_use_fp8(gate + 1)
+    assert not api.gate_use_fp8(1) and api.gate_use_fp8(1 << 20)
