@@ -64,6 +64,23 @@ int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d,
                      const float* scale_in, void* x_fp8, float* scale_out,
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The four quantizations of one ICL attention call in two launches instead of
+ * seven (same arithmetic and bit-identical results to four fp8attn_quantize
+ * calls): per-head absmax scales for Q_train, K and V (paper Eq. 2), and Q_test
+ * quantized with the train-query scale (Method section, shared query scale).  It
+ * removes most of the launch overhead that makes quantization dominate at small
+ * train-row counts (the paper's latency tables below ~8k rows).
+ *
+ *   q_train, k, v   in  bf16 [B,H,n_train,d]      q_test in bf16 [B,H,n_test,d] (NULL iff n_test == 0)
+ *   *_fp8           out e4m3, same shapes          scale_q/k/v out fp32 [B,H]
+ * n_train >= 1, n_test >= 0.
+ */
+int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
+                         int B, int H, int64_t n_train, int64_t n_test, int d,
+                         void* q_train_fp8, void* k_fp8, void* v_fp8, void* q_test_fp8,
+                         float* scale_q, float* scale_k, float* scale_v,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Fused FP8 ICL attention (paper Eq. 1 with the Method section's two-call
  * structure and quantization placement).
  *

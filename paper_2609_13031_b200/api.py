@@ -23,6 +23,7 @@ EXPORTS = (
     "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
+    "fp8attn_quantize_qkv",
 )
 TEST_ROWS_USE_KV_HEAD0 = 1
 GATE_TRAIN_ROWS = 8192
@@ -63,6 +64,9 @@ def load() -> ctypes.CDLL:
     lib.bf16attn_icl_forward_ex.restype = i32
     lib.bf16attn_icl_forward_ex.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, u32, vp, vp,
                                             vp, sz, vp]
+    lib.fp8attn_quantize_qkv.restype = i32
+    lib.fp8attn_quantize_qkv.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
+                                         vp, vp, vp, vp, sz, vp]
     lib.fp8attn_gate_use_fp8.restype = i32
     lib.fp8attn_gate_use_fp8.argtypes = [i64]
     lib.bf16attn_icl_forward.restype = i32
@@ -148,6 +152,28 @@ def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor
     return out, scale_out
 
 
+def quantize_qkv(q_train, k, v, q_test, workspace, out=None):
+    """fp8attn_quantize_qkv: all four quantizations of one attention call in two
+    launches.  Returns dict(q8, k8, v8, t8, sq, sk, sv); ``out`` may supply those
+    tensors preallocated."""
+    B, H, n_train, d = _dims(k)
+    n_test = 0 if q_test is None else q_test.shape[2]
+    dev = k.device
+    o = dict(out or {})
+    for name, rows in (("q8", n_train), ("k8", n_train), ("v8", n_train), ("t8", n_test)):
+        if name not in o:
+            o[name] = torch.empty((B, H, rows, d), dtype=torch.uint8, device=dev)
+    for name in ("sq", "sk", "sv"):
+        if name not in o:
+            o[name] = torch.empty((B, H), dtype=torch.float32, device=dev)
+    rc = load().fp8attn_quantize_qkv(
+        _ptr(q_train), _ptr(k), _ptr(v), _ptr(q_test) if n_test else None, B, H, n_train, n_test, d,
+        _ptr(o["q8"]), _ptr(o["k8"]), _ptr(o["v8"]), _ptr(o["t8"]) if n_test else None,
+        _ptr(o["sq"]), _ptr(o["sk"]), _ptr(o["sv"]), _ptr(workspace), workspace.numel(), _stream())
+    _check("fp8attn_quantize_qkv", rc)
+    return o
+
+
 def gate_use_fp8(n_train: int) -> bool:
     """fp8attn_gate_use_fp8: the paper's N > 8192 dispatch rule."""
     return bool(load().fp8attn_gate_use_fp8(int(n_train)))
@@ -221,10 +247,20 @@ def icl_attention(q_train, q_test, k, v, workspace=None, softmax_scale: float = 
     B, H, _, _ = _dims(k)
     if workspace is None:
         workspace = new_workspace(B, H, k.device)
-    q8, sq = quantize(q_train, workspace)
-    k8, sk = quantize(k, workspace)
-    v8, sv = quantize(v, workspace)
-    t8 = None
-    if q_test is not None and q_test.shape[2] > 0:
-        t8, _ = quantize(q_test, workspace, scale_in=sq)
+    has_test = q_test is not None and q_test.shape[2] > 0
+    o = quantize_qkv(q_train, k, v, q_test if has_test else None, workspace)
+    q8, k8, v8, sq, sk, sv = o["q8"], o["k8"], o["v8"], o["sq"], o["sk"], o["sv"]
+    t8 = o["t8"] if has_test else None
     return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale)
+
+
+def icl_attention_gated(q_train, q_test, k, v, workspace=None, softmax_scale: float = 0.0):
+    """The paper's final configuration: FP8 path only above the N > 8192 gate
+    (fp8attn_gate_use_fp8), the 16-bit path below it."""
+    B, H, n_train, _ = _dims(k)
+    if workspace is None:
+        workspace = new_workspace(B, H, k.device)
+    if gate_use_fp8(n_train):
+        return icl_attention(q_train, q_test, k, v, workspace, softmax_scale)
+    has_test = q_test is not None and q_test.shape[2] > 0
+    return icl_forward_bf16(q_train, q_test if has_test else None, k, v, workspace, softmax_scale)

@@ -11,14 +11,15 @@ namespace fp8attn {
 // Workspace layout (device memory, caller-owned, zero-filled once):
 //   [0,4)    device status word (fp8attn_status_t, 0 = ok); first error wins
 //   [4,8)    detail code of that error (which wait expired, which CTA)
-//   [256, 256 + 4*B*H)  per-(b,h) absmax accumulators (fp32 bit patterns) of the
-//                       quantizer; cleared at the start of every quantize call
+//   [256, 256 + 12*B*H) three sets of per-(b,h) absmax accumulators (fp32 bit
+//                       patterns): one is used by fp8attn_quantize, all three (Q, K, V)
+//                       by fp8attn_quantize_qkv; cleared at the start of every call
 constexpr size_t kWsStatusOffset = 0;
 constexpr size_t kWsDetailOffset = 4;
 constexpr size_t kWsAmaxOffset = 256;
 
 inline size_t workspace_bytes(int B, int H) {
-    size_t amax = (size_t)4 * (size_t)B * (size_t)H;
+    size_t amax = (size_t)12 * (size_t)B * (size_t)H;
     return kWsAmaxOffset + ((amax + 255) / 256) * 256;
 }
 
@@ -28,6 +29,11 @@ void count_launch();
 int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
                     const float* scale_in, void* x_fp8, float* scale_out,
                     uint32_t* amax_bits, cudaStream_t stream);
+
+int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
+                        int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
+                        void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
+                        float* scale_v, uint32_t* amax_bits, cudaStream_t stream);
 
 // attention.cu
 struct AttnParams {

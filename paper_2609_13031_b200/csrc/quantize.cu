@@ -29,9 +29,10 @@ __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) {
     return *reinterpret_cast<__nv_bfloat162*>(&u);
 }
 
-// grid: (blocks_per_head, n_heads).  A head is vecs_per_head 16-byte vectors.
-__global__ void __launch_bounds__(kThreads)
-absmax_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, uint32_t* __restrict__ amax_bits) {
+// One block's share of max |x| over head blockIdx.y (vecs_per_head 16-byte vectors),
+// merged into amax_bits[blockIdx.y].
+__device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t vecs_per_head,
+                                            uint32_t* __restrict__ amax_bits) {
     const uint4* xh = x + (int64_t)blockIdx.y * vecs_per_head;
     __nv_bfloat162 m = as_bf162(0u);
     int64_t stride = (int64_t)gridDim.x * kThreads;
@@ -71,6 +72,12 @@ absmax_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, uint32_t* __re
     }
 }
 
+// grid: (blocks_per_head, n_heads).
+__global__ void __launch_bounds__(kThreads)
+absmax_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, uint32_t* __restrict__ amax_bits) {
+    absmax_body(x, vecs_per_head, amax_bits);
+}
+
 // two floats -> two e4m3 codes (lo in bits 0..7, hi in bits 8..15), RNE, saturating
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
     uint16_t r;
@@ -87,12 +94,12 @@ __device__ __forceinline__ uint32_t quant4(uint32_t w0, uint32_t w1, float s) {
     return cvt_e4m3x2(a, b) | (cvt_e4m3x2(c, e) << 16);
 }
 
-// grid: (blocks_per_head, n_heads).  Each thread turns 32 B of bf16 into 16 B of
-// e4m3 per step.  pairs_per_head = elems_per_head / 16.
-__global__ void __launch_bounds__(kThreads)
-quantize_kernel(const uint4* __restrict__ x, int64_t pairs_per_head,
-                const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
-                uint4* __restrict__ out, float* __restrict__ scale_out) {
+// One block's share of head blockIdx.y.  Each thread turns 32 B of bf16 into 16 B
+// of e4m3 per step.  pairs_per_head = elems_per_head / 16.
+__device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64_t pairs_per_head,
+                                              const float* __restrict__ scale_in,
+                                              const uint32_t* __restrict__ amax_bits,
+                                              uint4* __restrict__ out, float* __restrict__ scale_out) {
     float s;
     if (scale_in != nullptr) {
         s = scale_in[blockIdx.y];
@@ -117,7 +124,69 @@ quantize_kernel(const uint4* __restrict__ x, int64_t pairs_per_head,
     }
 }
 
+// grid: (blocks_per_head, n_heads).
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const uint4* __restrict__ x, int64_t pairs_per_head,
+                const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
+                uint4* __restrict__ out, float* __restrict__ scale_out) {
+    quantize_body(x, pairs_per_head, scale_in, amax_bits, out, scale_out);
+}
+
+// All tensors of one attention call in two launches: blockIdx.z picks the tensor.
+struct QuantBatch {
+    const uint4* x[4];
+    uint4* out[4];
+    int64_t pairs_per_head[4];
+    const uint32_t* amax_in[4];   // accumulators the scale is derived from
+    uint32_t* amax_acc[4];        // accumulators this tensor's maximum goes to (NULL: none)
+    float* scale_out[4];
+};
+
+__global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch b) {
+    const int z = blockIdx.z;
+    if (b.amax_acc[z] != nullptr) absmax_body(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
+}
+
+__global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBatch b) {
+    const int z = blockIdx.z;
+    quantize_body(b.x[z], b.pairs_per_head[z], nullptr, b.amax_in[z], b.out[z], b.scale_out[z]);
+}
+
 }  // namespace
+
+int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
+                        int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
+                        void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
+                        float* scale_v, uint32_t* amax_bits, cudaStream_t stream) {
+    if (n_heads <= 0) return FP8ATTN_OK;
+    if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
+    QuantBatch b;
+    const void* xs[4] = {q_train, k, v, q_test};
+    void* outs[4] = {q_train_fp8, k_fp8, v_fp8, q_test_fp8};
+    float* scales[4] = {scale_q, scale_k, scale_v, nullptr};
+    for (int z = 0; z < 4; ++z) {
+        b.x[z] = static_cast<const uint4*>(xs[z]);
+        b.out[z] = static_cast<uint4*>(outs[z]);
+        b.pairs_per_head[z] = (z == 3 ? elems_test : elems_train) / 16;
+        // the test queries reuse the train-query maximum (slot 0): shared query scale
+        b.amax_in[z] = amax_bits + (z == 3 ? 0 : z) * n_heads;
+        b.amax_acc[z] = z == 3 ? nullptr : amax_bits + z * n_heads;
+        b.scale_out[z] = scales[z];
+    }
+    const int tensors = elems_test > 0 ? 4 : 3;
+    const int64_t want = (148 * 16 + n_heads * 3 - 1) / (n_heads * 3);
+    const int64_t have = (elems_train / 16 + kThreads - 1) / kThreads;
+    const unsigned bx = (unsigned)(want < have ? (want < 1 ? 1 : want) : (have < 1 ? 1 : have));
+    if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
+        return FP8ATTN_ERR_CUDA;
+    if (elems_train > 0) {
+        absmax_batch_kernel<<<dim3(bx, (unsigned)n_heads, 3), kThreads, 0, stream>>>(b);
+        count_launch();
+    }
+    quantize_batch_kernel<<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
+}
 
 int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
                     const float* scale_in, void* x_fp8, float* scale_out,

@@ -109,3 +109,24 @@ def test_argument_errors_are_reported_on_the_host():
     assert q(p(x), 1, 2, 4, 64, None, p(o), p(s), None, ws.numel(), None) == api.ERR_WORKSPACE
     assert q(p(x), 1, 2, 4, 64, None, p(o), p(s), p(ws), ws.numel(), None) == api.OK
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("cfg,n,m", [("C1", 512, 128), ("C2", 8192, 2048), ("C4", 3000, 0), ("C3", 4096, 1),
+                                      ("C5", 1, 0)])
+def test_fused_qkv_quantize_matches_oracle(cfg, n, m):
+    """fp8attn_quantize_qkv (two launches) is bit-identical to the oracle, including the
+    shared train-query scale for the test queries."""
+    w = W.CONFIGS[cfg].scaled(n, m)
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    o = api.quantize_qkv(to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]),
+                         to_dev(g["q_test"]) if m else None, ws)
+    rq, rsq = oracle.quantize(g["q_train"])
+    rk, rsk = oracle.quantize(g["k"])
+    rv, rsv = oracle.quantize(g["v"])
+    for got, ref in ((o["q8"], rq), (o["k8"], rk), (o["v8"], rv), (o["sq"], rsq), (o["sk"], rsk), (o["sv"], rsv)):
+        assert np.array_equal(got.cpu().numpy(), ref)
+    if m:
+        rt, _ = oracle.quantize(g["q_test"], scale_in=rsq)
+        assert np.array_equal(o["t8"].cpu().numpy(), rt)
+    assert api.last_device_status(ws) == (0, 0)
