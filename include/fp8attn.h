@@ -81,6 +81,21 @@ int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, cons
                          float* scale_q, float* scale_k, float* scale_v,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* fp8attn_quantize_qkv with a flags word.
+ * FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS: the query scale is the per-head absmax over
+ * the train AND the test queries (the single-call form the paper uses for
+ * TabICLv2, appendix: one attention call over all rows, quantized with per-head
+ * dynamic scales).  Test predictions then depend on the test batch.  Without
+ * the flag the scale comes from the train queries alone (the paper's proposal).
+ * The "per-call query scale" ablation arm needs no flag: quantize the test
+ * queries with fp8attn_quantize and scale_in = NULL. */
+#define FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS 1u
+int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test,
+                            int B, int H, int64_t n_train, int64_t n_test, int d,
+                            void* q_train_fp8, void* k_fp8, void* v_fp8, void* q_test_fp8,
+                            float* scale_q, float* scale_k, float* scale_v, uint32_t flags,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Fused FP8 ICL attention (paper Eq. 1 with the Method section's two-call
  * structure and quantization placement).
  *

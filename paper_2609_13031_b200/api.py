@@ -23,8 +23,9 @@ EXPORTS = (
     "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
-    "fp8attn_quantize_qkv",
+    "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex",
 )
+QUERY_SCALE_FROM_ALL_ROWS = 1
 TEST_ROWS_USE_KV_HEAD0 = 1
 GATE_TRAIN_ROWS = 8192
 
@@ -67,6 +68,9 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_quantize_qkv.restype = i32
     lib.fp8attn_quantize_qkv.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
                                          vp, vp, vp, vp, sz, vp]
+    lib.fp8attn_quantize_qkv_ex.restype = i32
+    lib.fp8attn_quantize_qkv_ex.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
+                                            vp, vp, vp, u32, vp, sz, vp]
     lib.fp8attn_gate_use_fp8.restype = i32
     lib.fp8attn_gate_use_fp8.argtypes = [i64]
     lib.bf16attn_icl_forward.restype = i32
@@ -152,7 +156,7 @@ def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor
     return out, scale_out
 
 
-def quantize_qkv(q_train, k, v, q_test, workspace, out=None):
+def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
     """fp8attn_quantize_qkv: all four quantizations of one attention call in two
     launches.  Returns dict(q8, k8, v8, t8, sq, sk, sv); ``out`` may supply those
     tensors preallocated."""
@@ -166,11 +170,15 @@ def quantize_qkv(q_train, k, v, q_test, workspace, out=None):
     for name in ("sq", "sk", "sv"):
         if name not in o:
             o[name] = torch.empty((B, H), dtype=torch.float32, device=dev)
-    rc = load().fp8attn_quantize_qkv(
-        _ptr(q_train), _ptr(k), _ptr(v), _ptr(q_test) if n_test else None, B, H, n_train, n_test, d,
-        _ptr(o["q8"]), _ptr(o["k8"]), _ptr(o["v8"]), _ptr(o["t8"]) if n_test else None,
-        _ptr(o["sq"]), _ptr(o["sk"]), _ptr(o["sv"]), _ptr(workspace), workspace.numel(), _stream())
-    _check("fp8attn_quantize_qkv", rc)
+    args = (_ptr(q_train), _ptr(k), _ptr(v), _ptr(q_test) if n_test else None, B, H, n_train, n_test, d,
+            _ptr(o["q8"]), _ptr(o["k8"]), _ptr(o["v8"]), _ptr(o["t8"]) if n_test else None,
+            _ptr(o["sq"]), _ptr(o["sk"]), _ptr(o["sv"]))
+    if flags:
+        rc = load().fp8attn_quantize_qkv_ex(*args, int(flags), _ptr(workspace), workspace.numel(), _stream())
+        _check("fp8attn_quantize_qkv_ex", rc)
+    else:
+        rc = load().fp8attn_quantize_qkv(*args, _ptr(workspace), workspace.numel(), _stream())
+        _check("fp8attn_quantize_qkv", rc)
     return o
 
 

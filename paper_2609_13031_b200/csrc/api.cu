@@ -90,13 +90,14 @@ int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d, cons
                            static_cast<cudaStream_t>(cuda_stream));
 }
 
-int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test, int B,
+int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test, int B,
                          int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
                          void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k, float* scale_v,
-                         void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+                         uint32_t flags, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS) return FP8ATTN_ERR_INVALID_ARG;
     if (!q_train || !k || !v || !q_train_fp8 || !k_fp8 || !v_fp8 || !scale_q || !scale_k || !scale_v)
         return FP8ATTN_ERR_INVALID_ARG;
     if (n_test > 0 && (!q_test || !q_test_fp8)) return FP8ATTN_ERR_INVALID_ARG;
@@ -110,7 +111,16 @@ int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, cons
     uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
     return launch_quantize_qkv(q_train, k, v, q_test, (int64_t)B * H, n_train * (int64_t)d,
                                n_test * (int64_t)d, q_train_fp8, k_fp8, v_fp8, q_test_fp8, scale_q, scale_k,
-                               scale_v, amax, static_cast<cudaStream_t>(cuda_stream));
+                               scale_v, amax, flags, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test, int B,
+                         int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
+                         void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k, float* scale_v,
+                         void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    return fp8attn_quantize_qkv_ex(q_train, k, v, q_test, B, H, n_train, n_test, d, q_train_fp8, k_fp8,
+                                   v_fp8, q_test_fp8, scale_q, scale_k, scale_v, 0u, workspace,
+                                   workspace_bytes_, cuda_stream);
 }
 
 int fp8attn_icl_forward(const void* q_train_fp8, const void* q_test_fp8, const void* k_fp8,

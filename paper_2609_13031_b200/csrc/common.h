@@ -33,7 +33,7 @@ int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
 int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
-                        float* scale_v, uint32_t* amax_bits, cudaStream_t stream);
+                        float* scale_v, uint32_t* amax_bits, uint32_t flags, cudaStream_t stream);
 
 // attention.cu
 struct AttnParams {

@@ -144,7 +144,8 @@ struct QuantBatch {
 
 __global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch b) {
     const int z = blockIdx.z;
-    if (b.amax_acc[z] != nullptr) absmax_body(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
+    if (b.amax_acc[z] != nullptr && b.pairs_per_head[z] > 0)
+        absmax_body(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
 }
 
 __global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBatch b) {
@@ -157,7 +158,7 @@ __global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBat
 int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
-                        float* scale_v, uint32_t* amax_bits, cudaStream_t stream) {
+                        float* scale_v, uint32_t* amax_bits, uint32_t flags, cudaStream_t stream) {
     if (n_heads <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     QuantBatch b;
@@ -171,6 +172,8 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
         // the test queries reuse the train-query maximum (slot 0): shared query scale
         b.amax_in[z] = amax_bits + (z == 3 ? 0 : z) * n_heads;
         b.amax_acc[z] = z == 3 ? nullptr : amax_bits + z * n_heads;
+        // single-call form: the query scale covers train and test queries alike
+        if (z == 3 && (flags & FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS) && elems_test > 0) b.amax_acc[z] = amax_bits;
         b.scale_out[z] = scales[z];
     }
     const int tensors = elems_test > 0 ? 4 : 3;
@@ -180,7 +183,7 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
     if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
         return FP8ATTN_ERR_CUDA;
     if (elems_train > 0) {
-        absmax_batch_kernel<<<dim3(bx, (unsigned)n_heads, 3), kThreads, 0, stream>>>(b);
+        absmax_batch_kernel<<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
         count_launch();
     }
     quantize_batch_kernel<<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);

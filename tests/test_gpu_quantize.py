@@ -130,3 +130,22 @@ def test_fused_qkv_quantize_matches_oracle(cfg, n, m):
         rt, _ = oracle.quantize(g["q_test"], scale_in=rsq)
         assert np.array_equal(o["t8"].cpu().numpy(), rt)
     assert api.last_device_status(ws) == (0, 0)
+
+
+def test_fused_qkv_query_scale_from_all_rows():
+    """Single-call form: one query scale over train and test queries together."""
+    w = W.CONFIGS["C2"].scaled(700, 900)
+    g = W.generate(w)
+    g["q_test"] = f32_to_bf16_bits(W.bf16_bits_to_f32(g["q_test"]) * np.float32(3.0))   # test rows set the maximum
+    ws = api.new_workspace(w.B, w.H)
+    o = api.quantize_qkv(to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]), to_dev(g["q_test"]), ws,
+                         flags=api.QUERY_SCALE_FROM_ALL_ROWS)
+    _, s_all = oracle.quantize(np.concatenate([g["q_train"], g["q_test"]], axis=2))
+    rq, _ = oracle.quantize(g["q_train"], scale_in=s_all)
+    rt, _ = oracle.quantize(g["q_test"], scale_in=s_all)
+    _, s_train = oracle.quantize(g["q_train"])
+    assert np.all(s_all > s_train)
+    assert np.array_equal(o["sq"].cpu().numpy(), s_all)
+    assert np.array_equal(o["q8"].cpu().numpy(), rq) and np.array_equal(o["t8"].cpu().numpy(), rt)
+    rk, rsk = oracle.quantize(g["k"])
+    assert np.array_equal(o["k8"].cpu().numpy(), rk) and np.array_equal(o["sk"].cpu().numpy(), rsk)
