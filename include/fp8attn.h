@@ -166,6 +166,28 @@ int bf16attn_icl_forward_ex(const void* q_train, const void* q_test, const void*
 #define FP8ATTN_GATE_TRAIN_ROWS 8192
 int fp8attn_gate_use_fp8(int64_t n_train);
 
+/* Seeded Gaussian perturbation of Q, K or V (paper appendix, Eq. 3: the noise
+ * experiment that replaces quantization by an explicit perturbation):
+ *
+ *   x~[b,h] = x[b,h] + epsilon * rho[b,h] * Z,   rho[b,h] = sqrt( mean over the head of x^2 ),
+ *   Z iid N(0,1), independent per head; the paper sweeps epsilon over {1..5} x 0.0265.
+ *
+ *   x_bf16 in bf16 [B,H,rows,d]; out_bf16 out, same shape (may alias x_bf16);
+ *   rho_out out fp32 [B,H] or NULL.
+ * Z is a pure function of (seed, stream_id, b*H+h, element index): a run is
+ * reproducible from the seed, and different stream_id values (one per tensor and
+ * layer, say) give independent fields.  Perturbing K and V once and passing the
+ * result to fp8attn_icl_forward / bf16attn_icl_forward is the paper's
+ * "coordinated" arm: both attention calls then consume the same noisy K, V.
+ * The normals come from Box-Muller in fp32 (hardware log / sin / cos), the sum of
+ * squares is accumulated in fp64; results agree with an fp64 evaluation to within
+ * one bf16 rounding step of the result (plus ~1e-6 of the two terms where they cancel).
+ */
+int fp8attn_perturb(const void* x_bf16, int B, int H, int64_t rows, int d,
+                    float epsilon, uint64_t seed, uint32_t stream_id,
+                    void* out_bf16, float* rho_out,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Allocation-free quantizer (the paper has no counterpart; this is a
  * packaging variant of fp8attn_quantize, same arithmetic, same results).
  *

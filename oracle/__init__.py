@@ -72,6 +72,11 @@ def _load():
                 ctypes.c_int]
             lib.oracle_icl_attention_rows.restype = None
             lib.oracle_icl_attention_rows.argtypes = [ctypes.POINTER(_AttnArgs)]
+            lib.oracle_perturb.restype = None
+            lib.oracle_perturb.argtypes = [
+                ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_int,
+                ctypes.c_double, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p,
+                ctypes.c_int]
             row_args = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
                         ctypes.c_float, ctypes.c_float, ctypes.c_int64,
                         ctypes.c_int64, ctypes.c_int, ctypes.c_double,
@@ -207,3 +212,18 @@ def lifted_p8_row(q, k, bh: int, row: int, sq: float = 1.0, sk: float = 1.0,
     """e4m3 codes of 2^8 * exp(t_j - max t) for one query row."""
     out = np.empty(k.shape[2], dtype=np.uint8)
     return _row_call(_load().oracle_lifted_p8_row, q, k, sq, sk, alpha, bh, row, out)
+
+
+# ---- Gaussian perturbation (Eq. 3) ---------------------------------------------
+
+def perturb(x_bf16_bits: np.ndarray, epsilon: float, seed: int, stream_id: int,
+            nthreads: int | None = None):
+    """bf16 bits [B,H,R,d] -> (perturbed bf16 bits, rho fp64 [B,H]):
+    x + epsilon * rho[b,h] * N(0,1), rho = per-head RMS."""
+    x = np.ascontiguousarray(x_bf16_bits, dtype=np.uint16)
+    B, H, R, d = x.shape
+    out = np.empty_like(x)
+    rho = np.zeros((B, H), dtype=np.float64)
+    _load().oracle_perturb(_ptr(x), B, H, R, d, float(epsilon), int(seed), int(stream_id),
+                           _ptr(out), _ptr(rho), nthreads or hardware_threads())
+    return out, rho

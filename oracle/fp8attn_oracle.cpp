@@ -338,4 +338,65 @@ void oracle_lifted_p8_row(const void* q, const void* k, int is_fp8,
         p8[j] = encode(std::ldexp(std::exp2((t[j] - m) * LOG2E), 8));
 }
 
+// ---- Gaussian perturbation (Eq. 3 of the appendix) ---------------------------
+// x~ = x + eps * rho * z per head, rho = sqrt(mean x^2), z ~ N(0,1).  The normal
+// field is the library's documented generator restated here in fp64: a 64-bit
+// mix of (seed, stream, head, element-pair index) gives two 32-bit uniforms
+// u1 = (hi + 1/2) / 2^32, u2 = (lo + 1/2) / 2^32, and Box-Muller gives
+// z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2).
+// The result is rounded once, from fp64, to the nearest bf16 (ties to even).
+static uint64_t perturb_mix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+static uint16_t double_to_bf16_bits(double v) {
+    // nearest bf16 to v: the two bf16 neighbours of |v| are compared in fp64
+    double a = std::fabs(v);
+    float f = (float)a;
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    uint32_t lo = u & 0xFFFF0000u;
+    float flo;
+    std::memcpy(&flo, &lo, 4);
+    if ((double)flo > a) { lo -= 0x10000u; std::memcpy(&flo, &lo, 4); }
+    uint32_t hi = lo + 0x10000u;
+    float fhi;
+    std::memcpy(&fhi, &hi, 4);
+    double dlo = a - (double)flo, dhi = (double)fhi - a;
+    uint32_t pick = dlo < dhi ? lo : (dhi < dlo ? hi : (((lo >> 16) & 1u) ? hi : lo));
+    return (uint16_t)((pick >> 16) | (std::signbit(v) ? 0x8000u : 0u));
+}
+
+void oracle_perturb(const uint16_t* x, int B, int H, int64_t R, int d, double eps, uint64_t seed,
+                    uint32_t stream_id, uint16_t* out, double* rho_out, int nthreads) {
+    const int64_t per_head = R * (int64_t)d;
+    const double two_pi = 6.283185307179586476925286766559;
+    parallel_for((int64_t)B * H, nthreads, [&](int64_t bh) {
+        const uint16_t* xs = x + bh * per_head;
+        uint16_t* os = out + bh * per_head;
+        double ss = 0.0;
+        for (int64_t i = 0; i < per_head; ++i) {
+            double v = (double)bf16_to_float(xs[i]);
+            ss += v * v;
+        }
+        const double rho = per_head > 0 ? std::sqrt(ss / (double)per_head) : 0.0;
+        if (rho_out) rho_out[bh] = rho;
+        const uint64_t key = perturb_mix64(perturb_mix64(perturb_mix64(seed) ^
+                                                         ((uint64_t)stream_id * 0xD6E8FEB86659FD93ull)) ^
+                                           (uint64_t)bh);
+        for (int64_t i = 0; i < per_head; ++i) {
+            const uint64_t pair = (uint64_t)(i >> 1);
+            const uint64_t h = perturb_mix64(key ^ (pair * 0x9E3779B97F4A7C15ull));
+            const double u1 = ((double)(h >> 32) + 0.5) / 4294967296.0;
+            const double u2 = ((double)(h & 0xFFFFFFFFull) + 0.5) / 4294967296.0;
+            const double r = std::sqrt(-2.0 * std::log(u1));
+            const double z = (i & 1) ? r * std::sin(two_pi * u2) : r * std::cos(two_pi * u2);
+            os[i] = double_to_bf16_bits((double)bf16_to_float(xs[i]) + eps * rho * z);
+        }
+    });
+}
+
 }  // extern "C"

@@ -23,7 +23,7 @@ EXPORTS = (
     "fp8attn_workspace_bytes", "fp8attn_last_device_status", "fp8attn_status_string",
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
-    "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex",
+    "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex", "fp8attn_perturb",
 )
 QUERY_SCALE_FROM_ALL_ROWS = 1
 TEST_ROWS_USE_KV_HEAD0 = 1
@@ -71,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_quantize_qkv_ex.restype = i32
     lib.fp8attn_quantize_qkv_ex.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
                                             vp, vp, vp, u32, vp, sz, vp]
+    lib.fp8attn_perturb.restype = i32
+    lib.fp8attn_perturb.argtypes = [vp, i32, i32, i64, i32, f32, ctypes.c_uint64, u32, vp, vp, vp, sz, vp]
     lib.fp8attn_gate_use_fp8.restype = i32
     lib.fp8attn_gate_use_fp8.argtypes = [i64]
     lib.bf16attn_icl_forward.restype = i32
@@ -180,6 +182,21 @@ def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
         rc = load().fp8attn_quantize_qkv(*args, _ptr(workspace), workspace.numel(), _stream())
         _check("fp8attn_quantize_qkv", rc)
     return o
+
+
+def perturb(x: torch.Tensor, epsilon: float, seed: int, stream_id: int, workspace: torch.Tensor,
+            out: torch.Tensor | None = None, rho_out: torch.Tensor | None = None):
+    """fp8attn_perturb: x + epsilon * rho[b,h] * N(0,1) per head (paper Eq. 3); returns (out, rho)."""
+    B, H, rows, d = _dims(x)
+    assert x.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty_like(x)
+    if rho_out is None:
+        rho_out = torch.empty((B, H), dtype=torch.float32, device=x.device)
+    rc = load().fp8attn_perturb(_ptr(x), B, H, rows, d, float(epsilon), int(seed), int(stream_id),
+                                _ptr(out), _ptr(rho_out), _ptr(workspace), workspace.numel(), _stream())
+    _check("fp8attn_perturb", rc)
+    return out, rho_out
 
 
 def gate_use_fp8(n_train: int) -> bool:

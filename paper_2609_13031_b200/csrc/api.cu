@@ -161,6 +161,23 @@ int bf16attn_icl_forward_ex(const void* q_train, const void* q_test, const void*
                    flags);
 }
 
+int fp8attn_perturb(const void* x_bf16, int B, int H, int64_t rows, int d, float epsilon, uint64_t seed,
+                    uint32_t stream_id, void* out_bf16, float* rho_out, void* workspace,
+                    size_t workspace_bytes_, void* cuda_stream) {
+    int rc = check_shape(B, H, d);
+    if (rc != FP8ATTN_OK) return rc;
+    if (rows < 0 || !(epsilon == epsilon)) return FP8ATTN_ERR_INVALID_ARG;
+    if (rows > 0 && (!x_bf16 || !out_bf16)) return FP8ATTN_ERR_INVALID_ARG;
+    if (!aligned(x_bf16, 16) || !aligned(out_bf16, 16) || !aligned(rho_out, 4)) return FP8ATTN_ERR_INVALID_ARG;
+    rc = check_workspace(workspace, workspace_bytes_, B, H);
+    if (rc != FP8ATTN_OK) return rc;
+    rc = check_device();
+    if (rc != FP8ATTN_OK) return rc;
+    double* sumsq = reinterpret_cast<double*>(static_cast<char*>(workspace) + kWsAmaxOffset);
+    return launch_perturb(x_bf16, (int64_t)B * H, rows * (int64_t)d, epsilon, seed, stream_id, out_bf16,
+                          rho_out, sumsq, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int fp8attn_gate_use_fp8(int64_t n_train) { return n_train > FP8ATTN_GATE_TRAIN_ROWS ? 1 : 0; }
 
 size_t fp8attn_workspace_bytes(int B, int H, int64_t, int64_t, int) {

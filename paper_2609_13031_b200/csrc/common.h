@@ -13,7 +13,8 @@ namespace fp8attn {
 //   [4,8)    detail code of that error (which wait expired, which CTA)
 //   [256, 256 + 12*B*H) three sets of per-(b,h) absmax accumulators (fp32 bit
 //                       patterns): one is used by fp8attn_quantize, all three (Q, K, V)
-//                       by fp8attn_quantize_qkv; cleared at the start of every call
+//                       by fp8attn_quantize_qkv; cleared at the start of every call.
+//                       fp8attn_perturb keeps its per-head sums of squares (fp64) here too.
 constexpr size_t kWsStatusOffset = 0;
 constexpr size_t kWsDetailOffset = 4;
 constexpr size_t kWsAmaxOffset = 256;
@@ -34,6 +35,11 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
                         float* scale_v, uint32_t* amax_bits, uint32_t flags, cudaStream_t stream);
+
+// perturb.cu
+int launch_perturb(const void* x_bf16, int64_t n_heads, int64_t elems_per_head, float epsilon,
+                   uint64_t seed, uint32_t stream_id, void* out_bf16, float* rho_out, double* sumsq,
+                   cudaStream_t stream);
 
 // attention.cu
 struct AttnParams {

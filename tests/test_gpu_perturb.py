@@ -1,0 +1,77 @@
+"""GPU parity: fp8attn_perturb (appendix Eq. 3) against the fp64 oracle.  The kernel
+draws the same counter-based normal field in fp32, so a result may differ from the
+oracle's by one bf16 rounding step where the sum lands next to a rounding boundary;
+everything else must be identical."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import bf16_bits_to_f64
+from paper_2609_13031_b200 import api
+from paper_2609_13031_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def bf16_ulp(x):
+    """spacing of bf16 at |x| (8 significant bits)"""
+    return 2.0 ** (np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -120))) - 7)
+
+
+@pytest.mark.parametrize("cfg,n,eps", [("C1", 512, 0.0265), ("C4", 3000, 5 * 0.0265), ("C3", 1001, 0.053),
+                                        ("C2", 1, 0.0265)])
+def test_matches_oracle_within_one_bf16_step(cfg, n, eps):
+    w = W.CONFIGS[cfg].scaled(n, 0)
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    for stream_id, name in ((0, "q_train"), (1, "k"), (2, "v")):
+        out, rho = api.perturb(to_dev(g[name]), eps, seed=w.seed + 100, stream_id=stream_id, workspace=ws)
+        ref, ref_rho = oracle.perturb(g[name], eps, w.seed + 100, stream_id)
+        assert np.allclose(rho.cpu().numpy(), ref_rho, rtol=2e-6)
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        gf, rf = bf16_bits_to_f64(got), bf16_bits_to_f64(ref)
+        # one bf16 step of the result, plus the fp32 evaluation error of the two terms where
+        # they cancel (the kernel's normals and the sum are fp32: ~1e-6 of each term)
+        x = bf16_bits_to_f64(g[name])
+        slack = 4e-6 * (np.abs(x) + eps * ref_rho[:, :, None, None] * 6.0)
+        assert np.all(np.abs(gf - rf) <= bf16_ulp(np.maximum(np.abs(gf), np.abs(rf))) * 1.0001 + slack)
+        assert np.mean(got == ref) > 0.995, np.mean(got == ref)
+    assert api.last_device_status(ws) == (0, 0)
+
+
+def test_zero_strength_identity_in_place_and_reproducible():
+    w = W.CONFIGS["C1"].scaled(300, 0)
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    x = to_dev(g["v"])
+    out, _ = api.perturb(x, 0.0, 1, 0, ws)
+    assert torch.equal(out, x)
+    a, _ = api.perturb(x, 0.1, 5, 7, ws)
+    b, _ = api.perturb(x, 0.1, 5, 7, ws)
+    assert torch.equal(a, b)
+    y = x.clone()
+    api.perturb(y, 0.1, 5, 7, ws, out=y)            # in place
+    assert torch.equal(y, a)
+    c, _ = api.perturb(x, 0.1, 5, 8, ws)
+    assert not torch.equal(a, c)
+
+
+def test_coordinated_noise_feeds_both_attention_calls():
+    """Perturbing K and V once and running the fused forward is the paper's coordinated arm:
+    a test query equal to a train query still gets that train row's output bit for bit."""
+    w = W.CONFIGS["C1"].scaled(384, 64)
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    k, _ = api.perturb(to_dev(g["k"]), 0.0265, 3, 1, ws)
+    v, _ = api.perturb(to_dev(g["v"]), 0.0265, 3, 2, ws)
+    q_train = to_dev(g["q_train"])
+    q_test = to_dev(g["q_test"]).clone()
+    q_test[:, :, 9] = q_train[:, :, 200]
+    o_tr, o_te = api.icl_forward_bf16(q_train, q_test, k, v, ws)
+    assert api.last_device_status(ws) == (0, 0)
+    assert torch.equal(o_te[:, :, 9], o_tr[:, :, 200])
