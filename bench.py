@@ -250,6 +250,7 @@ def main():
         torch.cuda.synchronize()
         if sampler.sm:
             break
+    preroll = (list(sampler.sm), set(sampler.reasons))
     sampler.sm.clear()
     sampler.reasons.clear()
     launches0 = api.launch_count()
@@ -268,6 +269,8 @@ def main():
     e_end.record()
     sync_all()
     launches = api.launch_count() - launches0
+    if not sampler.sm:                      # timed region shorter than one sampling period:
+        sampler.sm, sampler.reasons = preroll   # the samples of the untimed pre-roll under the same load
     clocks = sampler.result()
     total_ms = max_over_ranks(e_start.elapsed_time(e_end))
     ms_step = total_ms / args.steps
