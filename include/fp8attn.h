@@ -228,6 +228,16 @@ size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t n_test, in
  * receives a kernel-specific code saying which wait expired.  For tests. */
 int fp8attn_last_device_status(void* workspace, void* cuda_stream, uint32_t* detail);
 
+/* Self-test of the device-side error path (no counterpart in the paper).  Every
+ * wait inside the attention kernels is bounded; this launches one warp that
+ * waits, with a limit of limit_us microseconds (1..100000), on a barrier nothing
+ * ever signals, so the wait expires, FP8ATTN_ERR_TIMEOUT is recorded in the
+ * workspace and the kernel returns normally.  fp8attn_last_device_status() then
+ * reports it; until that call has cleared it, attention launches on the
+ * workspace do nothing.  The GPU context stays usable throughout. */
+int fp8attn_selftest_wait_timeout(void* workspace, size_t workspace_bytes, uint32_t limit_us,
+                                  void* cuda_stream);
+
 /* Static, human-readable name of a status code. */
 const char* fp8attn_status_string(int status);
 

@@ -24,6 +24,7 @@ EXPORTS = (
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
     "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex", "fp8attn_perturb",
+    "fp8attn_selftest_wait_timeout",
 )
 QUERY_SCALE_FROM_ALL_ROWS = 1
 TEST_ROWS_USE_KV_HEAD0 = 1
@@ -73,6 +74,8 @@ def load() -> ctypes.CDLL:
                                             vp, vp, vp, u32, vp, sz, vp]
     lib.fp8attn_perturb.restype = i32
     lib.fp8attn_perturb.argtypes = [vp, i32, i32, i64, i32, f32, ctypes.c_uint64, u32, vp, vp, vp, sz, vp]
+    lib.fp8attn_selftest_wait_timeout.restype = i32
+    lib.fp8attn_selftest_wait_timeout.argtypes = [vp, sz, u32, vp]
     lib.fp8attn_gate_use_fp8.restype = i32
     lib.fp8attn_gate_use_fp8.argtypes = [i64]
     lib.bf16attn_icl_forward.restype = i32
@@ -197,6 +200,12 @@ def perturb(x: torch.Tensor, epsilon: float, seed: int, stream_id: int, workspac
                                 _ptr(out), _ptr(rho_out), _ptr(workspace), workspace.numel(), _stream())
     _check("fp8attn_perturb", rc)
     return out, rho_out
+
+
+def selftest_wait_timeout(workspace: torch.Tensor, limit_us: int = 1000) -> None:
+    """fp8attn_selftest_wait_timeout: make one bounded device wait expire on purpose."""
+    rc = load().fp8attn_selftest_wait_timeout(_ptr(workspace), workspace.numel(), int(limit_us), _stream())
+    _check("fp8attn_selftest_wait_timeout", rc)
 
 
 def gate_use_fp8(n_train: int) -> bool:

@@ -178,6 +178,17 @@ int fp8attn_perturb(const void* x_bf16, int B, int H, int64_t rows, int d, float
                           rho_out, sumsq, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int fp8attn_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, uint32_t limit_us,
+                                  void* cuda_stream) {
+    if (limit_us == 0 || limit_us > 100000) return FP8ATTN_ERR_INVALID_ARG;
+    int rc = check_workspace(workspace, workspace_bytes_, 1, 1);
+    if (rc != FP8ATTN_OK) return rc;
+    rc = check_device();
+    if (rc != FP8ATTN_OK) return rc;
+    return launch_wait_timeout_selftest(reinterpret_cast<uint32_t*>(workspace), (uint64_t)limit_us * 1000ull,
+                                        static_cast<cudaStream_t>(cuda_stream));
+}
+
 int fp8attn_gate_use_fp8(int64_t n_train) { return n_train > FP8ATTN_GATE_TRAIN_ROWS ? 1 : 0; }
 
 size_t fp8attn_workspace_bytes(int B, int H, int64_t, int64_t, int) {

@@ -66,7 +66,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 // detail codes written next to FP8ATTN_ERR_TIMEOUT
 enum : uint32_t {
     kWaitQFull = 1, kWaitKFull, kWaitVFull, kWaitKEmpty, kWaitVEmpty, kWaitSFull, kWaitPFull, kWaitOFull,
-    kWaitSFree, kWaitPFree
+    kWaitSFree, kWaitPFree, kWaitSelfTest
 };
 
 template <bool kFp8, int kD>
@@ -113,6 +113,7 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 struct Waiter {
     uint32_t* status;
     bool dead;
+    uint64_t limit_ns = kWaitLimitNs;
     // kBackoffNs > 0: sleep that long between polls.  For waits with plenty of slack
     // (the TMA producer runs several stages ahead) this keeps the polling out of
     // the instruction queue that the softmax warps' MUFU and barrier traffic uses.
@@ -128,7 +129,7 @@ struct Waiter {
             }
             // another CTA already gave up: do not wait out the limit here as well
             if (*reinterpret_cast<volatile uint32_t*>(status) != 0u) { dead = true; return false; }
-            if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+            if (globaltimer_ns() - t0 > limit_ns) break;
         }
         dead = true;
         if (atomicCAS(status, 0u, (uint32_t)FP8ATTN_ERR_TIMEOUT) == 0u)
@@ -739,6 +740,20 @@ int launch(const AttnParams& p, cudaStream_t stream) {
 
 }  // namespace
 
+// Exercises the error path of the bounded waits without touching any real work:
+// one warp waits, with the given limit, on a barrier that nothing ever arrives on,
+// records the timeout in the status words and returns normally.
+__global__ void wait_timeout_selftest_kernel(uint32_t* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    Waiter w{status, false, limit_ns};
+    w.wait(smem_u32(&bar), 0, kWaitSelfTest);
+}
+
 #ifdef FP8ATTN_TRACE
 // Debug build only: where the kernels of CTA 0 write their clock stamps
 // (16 steps x 32 slots of int64), or NULL to switch tracing off.
@@ -747,6 +762,12 @@ extern "C" int fp8attn_debug_set_trace(void* device_buffer) {
     return cudaMemcpyToSymbol(g_trace_buf, &p, sizeof(p)) == cudaSuccess ? 0 : 4;
 }
 #endif
+
+int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
+}
 
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {
     if (fp8) return p.d == 64 ? launch<true, 64>(p, stream) : launch<true, 128>(p, stream);

@@ -52,5 +52,6 @@ struct AttnParams {
     uint32_t* status;  // workspace status words
 };
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream);
+int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
 
 }  // namespace fp8attn
