@@ -296,21 +296,64 @@ def main():
         ms_bf16 = max_over_ranks(a.elapsed_time(b)) / n_bf
 
     # ---- end to end: pinned host inputs -> device -> path -> host outputs, every step ----
-    def e2e_step():
-        for k in host:
-            dev[k].copy_(host[k], non_blocking=True)
-        quantize_all()
-        attention_fp8()
-        host_out["o_tr"].copy_(buf["o_tr"], non_blocking=True)
-        host_out["o_te"].copy_(buf["o_te"], non_blocking=True)
+    # Every step copies its own inputs from pinned host memory and its own results back.  The
+    # copies of neighbouring steps overlap the compute of the current one: three streams
+    # (copy-in, compute, copy-out) and two sets of device buffers, ordered by events.
+    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    sets = []
+    for _ in range(2):
+        d_in = {k: torch.empty_like(v, device="cuda") for k, v in host.items()}
+        d_buf = {k: torch.empty_like(v) for k, v in buf.items()}
+        sets.append((d_in, d_buf))
+    free_in = [None, None]      # event: compute no longer reads this input set
+    free_out = [None, None]     # event: copy-out no longer reads this output set
 
-    e2e_step()
+    def e2e_run(n):
+        for i in range(n):
+            d_in, d_buf = sets[i % 2]
+            with torch.cuda.stream(s_in):
+                if free_in[i % 2] is not None:
+                    s_in.wait_event(free_in[i % 2])
+                for k in host:
+                    d_in[k].copy_(host[k], non_blocking=True)
+                e_in = torch.cuda.Event()
+                e_in.record(s_in)
+            with torch.cuda.stream(s_cmp):
+                s_cmp.wait_event(e_in)
+                if free_out[i % 2] is not None:
+                    s_cmp.wait_event(free_out[i % 2])
+                api.quantize_qkv(d_in["q_train"], d_in["k"], d_in["v"], d_in["q_test"], ws, out=d_buf)
+                api.icl_forward_fp8(d_buf["q8"], d_buf["t8"], d_buf["k8"], d_buf["v8"], d_buf["sq"],
+                                    d_buf["sk"], d_buf["sv"], ws, 0.0, out_train=d_buf["o_tr"],
+                                    out_test=d_buf["o_te"])
+                e_c = torch.cuda.Event()
+                e_c.record(s_cmp)
+                free_in[i % 2] = e_c
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(e_c)
+                host_out["o_tr"].copy_(d_buf["o_tr"], non_blocking=True)
+                host_out["o_te"].copy_(d_buf["o_te"], non_blocking=True)
+                e_o = torch.cuda.Event()
+                e_o.record(s_out)
+                free_out[i % 2] = e_o
+
+    def join_streams():
+        cur = torch.cuda.current_stream()
+        for st in (s_in, s_cmp, s_out):
+            cur.wait_stream(st)
+
+    for st in (s_in, s_cmp, s_out):
+        st.wait_stream(torch.cuda.current_stream())
+    e2e_run(2)
+    join_streams()
     sync_all()
-    n_e2e = max(2, min(args.steps, 5))
+    n_e2e = max(4, min(args.steps, 20))
     a, b = ev(), ev()
     a.record()
-    for _ in range(n_e2e):
-        e2e_step()
+    for st in (s_in, s_cmp, s_out):
+        st.wait_stream(torch.cuda.current_stream())
+    e2e_run(n_e2e)
+    join_streams()
     b.record()
     sync_all()
     ms_e2e = max_over_ranks(a.elapsed_time(b)) / n_e2e
