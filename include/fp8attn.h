@@ -21,7 +21,8 @@
  *     fp8attn_last_device_status(); the kernels never trap or spin forever.  A
  *     recorded device error is sticky: attention launches on that workspace do
  *     nothing until fp8attn_last_device_status() has read and cleared it.
- *   - Supported head dims: d = 64 and d = 128.  n_train >= 1, n_test >= 0.
+ *   - Supported head dims: d = 64 and d = 128.  n_train >= 1, n_test >= 0, each
+ *     below 2^31 - 256; B*H <= 65535.
  */
 #ifndef FP8ATTN_H_
 #define FP8ATTN_H_

@@ -194,3 +194,32 @@ def test_forward_argument_errors():
     assert f(*args(wsb=16)) == api.ERR_WORKSPACE
     assert f(*args()) == api.OK
     assert api.last_device_status(ws) == (0, 0)
+
+
+# ---- degenerate inputs ------------------------------------------------------------------
+
+def test_fp8_degenerate_heads_zero_queries_zero_keys_and_saturated_test_queries():
+    """Head 0: all-zero queries (uniform weights -> mean of the value rows); head 1: all-zero
+    keys (same); test queries far outside the train range saturate at +-448 and still match."""
+    w = W.CONFIGS["C1"].scaled(333, 50)
+    g = W.generate(w)
+    g["q_train"][:, 0] = 0
+    g["q_test"][:, 0] = 0
+    g["k"][:, 1] = 0
+    big = W.bf16_bits_to_f32(g["q_test"][:, 1]) * np.float32(50.0)      # beyond the train-query absmax
+    g["q_test"][:, 1] = f32_to_bf16_bits(big)
+    z = oracle_quantized(g)
+    assert np.all(z["sq"][:, 0] == 1.0) and np.all(z["sk"][:, 1] == 1.0)
+    assert (z["t8"][:, 1] & 0x7F).max() == 0x7E
+    o_tr, o_te = gpu_fp8_forward(z, w)
+    tab = oracle.e4m3_decode_table()
+    vhat = tab[z["v8"]] * z["sv"][:, :, None, None].astype(np.float64)
+    for out in (o_tr, o_te):
+        got = out_to_f64(out)
+        for h in (0, 1):
+            mean_v = vhat[0, h].mean(axis=0)
+            assert np.max(np.abs(got[0, h] - mean_v)) < 2e-2 * max(1.0, np.abs(mean_v).max()) + 5e-3
+    for name, out, q8, nq in (("train", o_tr, z["q8"], w.n_train), ("test", o_te, z["t8"], w.n_test)):
+        A, Abs, Bnd = oracle.icl_attention_rows(q8, z["k8"], z["v8"], np.arange(nq), sq=z["sq"], sk=z["sk"],
+                                                sv=z["sv"])
+        check_fp8_attention(out_to_f64(out), A, Abs, Bnd, diffuse=False, label=name, named_config=False)
