@@ -9,11 +9,8 @@
 //   warps 10-11 issue the P V tcgen05.mma of tile 0 and tile 1
 // Q K^T and P V are issued from different warps because a single warp cannot
 // issue tcgen05 instructions of this size fast enough to keep the tensor core fed.
-// Build options (compile-time, for experiments): FP8ATTN_SPLIT=2 lets two threads
-// share a row (16 softmax warps; they exchange partial maxima through shared memory
-// once per step), FP8ATTN_PINGPONG=1 makes the two tiles take strict turns on the
-// exponential phase, FP8ATTN_POLY_EVERY sets the share of exponentials computed by
-// a polynomial on the FMA pipe instead of the MUFU.
+// Build option: FP8ATTN_POLY_EVERY sets the share of exponentials computed by a
+// polynomial on the FMA pipe instead of the MUFU.
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
@@ -40,23 +37,14 @@ constexpr int kTileM = 128;           // query rows per tile
 #ifndef FP8ATTN_POLY_EVERY
 #define FP8ATTN_POLY_EVERY 2
 #endif
-#ifndef FP8ATTN_PINGPONG
-#define FP8ATTN_PINGPONG 0
-#endif
-#ifndef FP8ATTN_SPLIT
-#define FP8ATTN_SPLIT 1
-#endif
-// kSplit threads share a query row, each owning 1/kSplit of the key columns of a step.
-constexpr int kSplit = FP8ATTN_SPLIT;
-static_assert(kSplit == 1 || kSplit == 2, "row split");
-constexpr int kSoftmaxWarps = 8 * kSplit;
-constexpr int kQkWarp = kSoftmaxWarps, kTmaWarp = kSoftmaxWarps + 1, kPvWarp0 = kSoftmaxWarps + 2;
-constexpr int kNumThreads = (kSoftmaxWarps + 4) * 32;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kQkWarp = 8, kTmaWarp = 9, kPvWarp0 = 10;
+constexpr int kNumThreads = 12 * 32;
 // Register budgets after setmaxnreg.  The CTA's register pool is what it was
-// launched with (threads x launch registers); setmaxnreg.inc waits in hardware
+// launched with (384 threads x 168 registers); setmaxnreg.inc waits in hardware
 // until the pool can serve it, so the budgets must fit in it.
-constexpr int kLaunchRegs = kSplit == 2 ? 96 : 168;
-constexpr int kRegsSoftmax = kSplit == 2 ? 104 : 224;
+constexpr int kLaunchRegs = 168;
+constexpr int kRegsSoftmax = 224;
 constexpr int kRegsOther = 56;
 static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kNumThreads * kLaunchRegs,
               "setmaxnreg budgets exceed the CTA's register pool");
@@ -99,7 +87,7 @@ struct Cfg {
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], s_free[2], p_full[2], p_free[2], o_full[2];
+    uint64_t s_full[2], p_free[2], o_full[2];
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -262,7 +250,7 @@ __device__ long long* g_trace_buf;
 #define FP8ATTN_TRACE_INIT() long long* const trace_buf = (blockIdx.x == 0) ? g_trace_buf : nullptr
 #define FP8ATTN_STAMP(slot, j)                                                         \
     do {                                                                               \
-        if (trace_buf != nullptr && lane == 0 && (warp >= kSoftmaxWarps || (warp % (4 * kSplit)) == 0) && (j) >= 64 && (j) < 80)                \
+        if (trace_buf != nullptr && lane == 0 && (warp >= kSoftmaxWarps || (warp & 3) == 0) && (j) >= 64 && (j) < 80)                \
             trace_buf[((j) - 64) * 32 + (slot)] = clock64();                           \
     } while (0)
 #else
@@ -293,12 +281,11 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) 
     else tmem_st_x32(taddr, r);
 }
 
-// Named barriers (hardware-blocking, no polling).  1..8: the two warps sharing
-// rows when a row is split; 9, 10: whose turn the exponential phase is;
-// 11 + t: "S_t is in registers" (softmax -> Q K^T issuer); 13 + t: "P_t is in
-// tensor memory" (softmax -> P V issuer of tile t).
-constexpr uint32_t kTurnBarrier0 = 9, kSFreeBarrier0 = 11, kPFullBarrier0 = 13;
-constexpr uint32_t kSignalThreads = 128 * kSplit + 32;   // one tile's softmax threads + the issuer warp
+// Named barriers (hardware-blocking, no polling), one of each per query tile t:
+//   kSFreeBarrier0 + t  "S_t is in registers"        softmax warps -> Q K^T issuer
+//   kPFullBarrier0 + t  "P_t is in tensor memory"    softmax warps -> P V issuer of tile t
+constexpr uint32_t kSFreeBarrier0 = 1, kPFullBarrier0 = 3;
+constexpr uint32_t kSignalThreads = 128 + 32;   // one tile's softmax threads + the issuer warp
 
 struct KernelArgs {
     const float* scale_q; const float* scale_k; const float* scale_v;
@@ -322,7 +309,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ uint32_t tmem_slot;
-    __shared__ float xchg[2][2][2][kTileM];   // [step parity][tile][column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -359,8 +345,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.s_free[t]), 4 * kSplit);
-            mbar_init(smem_u32(&bars.p_full[t]), 4 * kSplit);
             mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
         }
@@ -501,18 +485,13 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     } else {
         // ========================= softmax + epilogue =========================
         setmaxnreg_inc<kRegsSoftmax>();
-        constexpr int kCols = kKeys / kSplit;          // key columns of a step owned by one thread
-        constexpr int kPColsT = C::kPCols / kSplit;    // P columns owned by one thread
-        constexpr int kOCols = kD / kSplit;            // output columns owned by one thread
-        const int t = warp / (4 * kSplit);             // query tile
-        const int h = (warp >> 2) % kSplit;            // which part of the columns
+        const int t = warp >> 2;                       // query tile
         if (t < ntiles) {
             const int row_in_tile = (warp & 3) * 32 + lane;
-            const uint32_t pair_barrier = 1 + t * 4 + (warp & 3);   // the warps that share rows
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0) + h * kCols;
-            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0) + h * kPColsT;
-            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD + h * kOCols;
+            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0);
+            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0);
+            const uint32_t tO = tmem + lane_addr + C::kColO + t * kD;
             float c = (args.softmax_scale > 0.f ? args.softmax_scale : rsqrtf((float)kD)) *
                       1.4426950408889634f;
             float sv_scale = 1.0f;
@@ -528,50 +507,36 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             float m = -INFINITY;
             uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // partial row sums
             constexpr uint32_t kNegInf = 0xff800000u;
-            // The two query tiles take turns on the exponential phase (tile 0 of step j,
-            // tile 1 of step j, tile 0 of step j+1, ...): one tile's MUFU work then runs
-            // under the other's tensor-memory loads, maximum and barrier traffic instead
-            // of both queueing on the MUFU at once and leaving it idle together.
-            const bool ping_pong = FP8ATTN_PINGPONG && ntiles == 2;
-            constexpr uint32_t kTurnThreads = 2 * 128 * kSplit;
-            if (ping_pong && t == 1) named_barrier_arrive(kTurnBarrier0, kTurnThreads);
             for (int j = 0; j < nkv; ++j) {
                 w.wait(smem_u32(&bars.s_full[t]), j & 1, kWaitSFull);
                 tc_fence_after_sync();
                 FP8ATTN_STAMP(t * 8 + 0, j);
-                // ---- this thread's part of the score row into registers ----
-                uint32_t s[kCols];
-                tmem_ld_cols<kCols>(tS, s);
-                tmem_wait_ld_cols<kCols>(s);
+                // ---- the whole score row of this thread into registers ----
+                uint32_t s[kKeys];
+                tmem_ld_cols<kKeys>(tS, s);
+                tmem_wait_ld_cols<kKeys>(s);
                 if (C::kSepP && j + 1 < nkv) {
                     // S may be overwritten by the next Q K^T from here on
                     tc_fence_before_sync();
                     named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
                 }
                 FP8ATTN_STAMP(t * 8 + 1, j);
-                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys) - h * kCols;
-                if (valid < kCols) {
+                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys);
+                if (valid < kKeys) {
 #pragma unroll
-                    for (int i = 0; i < kCols; ++i)
+                    for (int i = 0; i < kKeys; ++i)
                         if (i >= valid) s[i] = kNegInf;
                 }
-                // ---- row maximum (own columns, then the partner's through shared memory) ----
+                // ---- row maximum of the raw scores ----
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < kCols; i += 8) {
+                for (int i = 0; i < kKeys; i += 8) {
                     mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
                     mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
                     mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
                     mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
                 }
-                float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                if (kSplit == 2) {
-                    xchg[j & 1][t][h][row_in_tile] = m_tile;
-                    FP8ATTN_STAMP(t * 8 + 5, j);
-                    named_barrier_sync(pair_barrier, 64);
-                    FP8ATTN_STAMP(t * 8 + 6, j);
-                    m_tile = fmaxf(m_tile, xchg[j & 1][t][h ^ 1][row_in_tile]);
-                }
+                const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
                 // The reference maximum is the exact running maximum: the row maximum of
                 // the keys seen so far maps to 2^lift.
                 const float m_new = fmaxf(m, m_tile);
@@ -590,7 +555,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     l2a = mul2(l2a, ff);
                     l2b = mul2(l2b, ff);
 #pragma unroll
-                    for (int q = 0; q < kOCols / 16; ++q) {
+                    for (int q = 0; q < kD / 16; ++q) {
                         uint32_t o[16];
                         tmem_ld_x16(tO + q * 16, o);
                         tmem_wait_ld_x16(o);
@@ -602,18 +567,14 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 m = m_new;
                 const float nb = lift - m * c;
                 const uint64_t nbnb = pack2(nb, nb);
-                if (ping_pong) named_barrier_sync(kTurnBarrier0 + t, kTurnThreads);
                 FP8ATTN_STAMP(t * 8 + 2, j);
                 // ---- p = 2^(c*s - c*m + lift), row sums, P tile into tensor memory ----
-                // chunks of 32 keys (a last one of 16 where the column count asks for it)
 #pragma unroll
-                for (int k0 = 0; k0 < kCols; k0 += 32) {
+                for (int k0 = 0; k0 < kKeys; k0 += 32) {
                     constexpr int kPPer32 = kFp8 ? 8 : 16;
                     uint32_t p[kPPer32];
-                    const int n = (kCols - k0) < 32 ? (kCols - k0) : 32;
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
-                        if (i >= n) break;
                         const uint32_t* cur = s + k0 + i;
                         const uint64_t xa = fma2(pack2(__uint_as_float(cur[0]), __uint_as_float(cur[1])), cc, nbnb);
                         const uint64_t xb = fma2(pack2(__uint_as_float(cur[2]), __uint_as_float(cur[3])), cc, nbnb);
@@ -642,39 +603,31 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                     }
-                    if (n == 32) tmem_st_cols<kPPer32>(tP + (k0 / 32) * kPPer32, p);
-                    else tmem_st_cols<kPPer32 / 2>(tP + (k0 / 32) * kPPer32, p);
+                    tmem_st_cols<kPPer32>(tP + (k0 / 32) * kPPer32, p);
                 }
-                if (ping_pong) named_barrier_arrive(kTurnBarrier0 + (t ^ 1), kTurnThreads);
                 FP8ATTN_STAMP(t * 8 + 3, j);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 named_barrier_arrive(kPFullBarrier0 + t, kSignalThreads);
                 FP8ATTN_STAMP(t * 8 + 4, j);
             }
-            if (ping_pong && t == 0) named_barrier_sync(kTurnBarrier0, kTurnThreads);   // last turn token
-            // ---- row sum (plus the partner's) ----
+            // ---- row sum ----
             float l;
             {
                 float a0, a1, b0, b1;
                 unpack2(l2a, a0, a1);
                 unpack2(l2b, b0, b1);
                 l = (a0 + a1) + (b0 + b1);
-                if (kSplit == 2) {
-                    xchg[nkv & 1][t][h][row_in_tile] = l;
-                    named_barrier_sync(pair_barrier, 64);
-                    l += xchg[nkv & 1][t][h ^ 1][row_in_tile];
-                }
             }
-            // ---- epilogue: out = s_v * O / l, this thread's share of the columns ----
+            // ---- epilogue: out = s_v * O / l ----
             w.wait(smem_u32(&bars.o_full[t]), 0, kWaitOFull);
             tc_fence_after_sync();
             const int64_t row = row0 + t * kTileM + row_in_tile;
             const float inv = sv_scale / l;
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
-                                 ((int64_t)bh * q_rows + row) * kD + h * kOCols;
+                                 ((int64_t)bh * q_rows + row) * kD;
 #pragma unroll
-            for (int q = 0; q < kOCols / 32; ++q) {
+            for (int q = 0; q < kD / 32; ++q) {
                 uint32_t o[32];
                 tmem_ld_x32(tO + q * 32, o);
                 tmem_wait_ld_x32(o);
