@@ -79,6 +79,11 @@ struct Cfg {
     static constexpr uint32_t kColS0 = 0, kColS1 = kKeys, kColO = 256;
     static constexpr uint32_t kColP0 = !kSepP ? kColS0 : (kD == 128 ? 192u : 384u);
     static constexpr uint32_t kColP1 = !kSepP ? kColS1 : (kD == 128 ? 224u : 384u + 64u);
+    // Where tensor memory has room, P alternates between two buffers per tile (the second
+    // kPCols columns after the first), so that writing P of one step never waits for the
+    // P V of the step before.
+    static constexpr int kPBufs = (kFp8 && kD == 64) ? 2 : 1;
+    static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= (kD == 128 ? 32 : 64)), "TMEM layout");
     static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
     static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
     static constexpr size_t kSmemBytes = (size_t)2 * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
@@ -472,7 +477,9 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
 #pragma unroll
                     for (int kk = 0; kk < kKeys / C::kUmmaK; ++kk) {
                         const uint64_t b = b0 + (uint64_t)((kk * C::kUmmaK * C::kBoxBytes) >> 4);
-                        mma_ts<kFp8>(d, a + kk * 8, b, C::kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                        const uint32_t pa = (uint32_t)((C::kPBufs == 2 ? (j & 1) * C::kPCols : 0) + kk * 8);
+                        mma_ts<kFp8>(d, a + pa, b, C::kIdescPV,
+                                     (j > 0 || kk > 0) ? 1u : 0u);
                     }
                     mma_commit(smem_u32(&bars.p_free[t]));
                     mma_commit(smem_u32(&bars.v_empty[sv]));
@@ -542,6 +549,12 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 const float m_new = fmaxf(m, m_tile);
                 // P V of the previous step must be done before O is rescaled or P rewritten
                 bool pv_done = !(C::kSepP && j > 0);
+                if (C::kPBufs == 1 && !pv_done && !w.dead) {
+                    // ask now, use the answer a chunk of exponentials later: the usual case
+                    // (P V long done) then costs no stall in the middle of the chunk
+                    pv_done = mbar_test_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1);
+                    tc_fence_after_sync();
+                }
                 if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
                     FP8ATTN_STAMP(t * 8 + 7, j);
                     if (!pv_done) {
@@ -599,13 +612,21 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                             p[i / 2 + 1] = pack_bf16x2(p2, p3);
                         }
                     }
-                    if (k0 == 0 && !pv_done) {
+                    if (C::kPBufs == 1 && k0 == 0 && !pv_done) {
+                        FP8ATTN_STAMP(t * 8 + 5, j);
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
+                        FP8ATTN_STAMP(t * 8 + 6, j);
                     }
-                    tmem_st_cols<kPPer32>(tP + (k0 / 32) * kPPer32, p);
+                    tmem_st_cols<kPPer32>(tP + (uint32_t)((C::kPBufs == 2 ? (j & 1) * C::kPCols : 0) + (k0 / 32) * kPPer32), p);
                 }
                 FP8ATTN_STAMP(t * 8 + 3, j);
+                if (C::kPBufs == 2 && !pv_done) {
+                    // P V of the previous step has had this whole step to finish; once it
+                    // has, the buffer that the NEXT step writes (the one it read) is free.
+                    // That write comes after the next step's fence behind its wait for S.
+                    w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                }
                 tmem_wait_st();
                 tc_fence_before_sync();
                 named_barrier_arrive(kPFullBarrier0 + t, kSignalThreads);
