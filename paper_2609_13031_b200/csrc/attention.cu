@@ -9,8 +9,8 @@
 //   warps 10-11 issue the P V tcgen05.mma of tile 0 and tile 1
 // Q K^T and P V are issued from different warps because a single warp cannot
 // issue tcgen05 instructions of this size fast enough to keep the tensor core fed.
-// Build option: FP8ATTN_POLY_EVERY sets the share of exponentials computed by a
-// polynomial on the FMA pipe instead of the MUFU.
+// A share of the exponentials (Cfg::kPolyPer16 pairs of every 16) is computed by a
+// polynomial on the FMA pipe instead of the MUFU; FP8ATTN_POLY16 overrides it at build time.
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
@@ -34,9 +34,6 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileM = 128;           // query rows per tile
-#ifndef FP8ATTN_POLY_EVERY
-#define FP8ATTN_POLY_EVERY 2
-#endif
 constexpr int kSoftmaxWarps = 8;
 constexpr int kQkWarp = 8, kTmaWarp = 9, kPvWarp0 = 10;
 constexpr int kNumThreads = 12 * 32;
@@ -83,6 +80,12 @@ struct Cfg {
     // kPCols columns after the first), so that writing P of one step never waits for the
     // P V of the step before.
     static constexpr int kPBufs = (kFp8 && kD == 64) ? 2 : 1;
+    // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
+#ifdef FP8ATTN_POLY16
+    static constexpr int kPolyPer16 = FP8ATTN_POLY16;
+#else
+    static constexpr int kPolyPer16 = kFp8 ? (kD == 128 ? 8 : 4) : (kD == 128 ? 6 : 2);
+#endif
     static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= (kD == 128 ? 32 : 64)), "TMEM layout");
     static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
     static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
@@ -507,9 +510,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 sv_scale = args.scale_v[bh_kv];
             }
             const float lift = kFp8 ? 8.0f : 0.0f;
-            // every kPolyEvery-th group of four columns computes two of its exponentials
-            // with the polynomial (0 = never): 1 -> 50 %, 2 -> 25 %, 4 -> 12.5 % of all
-            constexpr int kPolyEvery = FP8ATTN_POLY_EVERY;
             const uint64_t cc = pack2(c, c);
             float m = -INFINITY;
             uint64_t l2a = pack2(0.f, 0.f), l2b = pack2(0.f, 0.f);   // partial row sums
@@ -594,10 +594,17 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         float p0, p1, p2, p3, x0, x1, x2, x3;
                         unpack2(xa, x0, x1);
                         unpack2(xb, x2, x3);
-                        p0 = ex2(x0);
-                        p1 = ex2(x1);
-                        if (kPolyEvery > 0 && ((i / 4) % kPolyEvery) == kPolyEvery - 1) {
-                            // this pair goes to the FMA pipe to take load off the MUFU
+                        // pair q of the chunk goes to the FMA pipe if the running count
+                        // q * kPolyPer16 / 16 steps up there: an even spread over the chunk
+                        constexpr int kPP = C::kPolyPer16;
+                        const int qa = i / 2, qb = i / 2 + 1;
+                        if (((qa + 1) * kPP) / 16 != (qa * kPP) / 16) {
+                            exp2_poly2<!kFp8>(pack2(fmaxf(x0, -120.f), fmaxf(x1, -120.f)), p0, p1);
+                        } else {
+                            p0 = ex2(x0);
+                            p1 = ex2(x1);
+                        }
+                        if (((qb + 1) * kPP) / 16 != (qb * kPP) / 16) {
                             exp2_poly2<!kFp8>(pack2(fmaxf(x2, -120.f), fmaxf(x3, -120.f)), p2, p3);
                         } else {
                             p2 = ex2(x2);
