@@ -80,11 +80,12 @@ struct Cfg {
     // kPCols columns after the first), so that writing P of one step never waits for the
     // P V of the step before.
     static constexpr int kPBufs = (kFp8 && kD == 64) ? 2 : 1;
+    static constexpr bool kLateRescale = kD == 128;             // O rescale at the end of the step
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
 #ifdef FP8ATTN_POLY16
     static constexpr int kPolyPer16 = FP8ATTN_POLY16;
 #else
-    static constexpr int kPolyPer16 = kFp8 ? (kD == 128 ? 8 : 4) : (kD == 128 ? 6 : 2);
+    static constexpr int kPolyPer16 = kFp8 ? 4 : (kD == 128 ? 8 : 2);
 #endif
     static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= (kD == 128 ? 32 : 64)), "TMEM layout");
     static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
@@ -555,26 +556,35 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     pv_done = mbar_test_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1);
                     tc_fence_after_sync();
                 }
-                if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
+                // Where the maximum moved for some row of this warp, l is rescaled now.  O is
+                // rescaled now too (kLateRescale false), or at the end of the step: by then
+                // the score registers are free, so the O columns go through registers in
+                // pipelined halves instead of dependent 16-column round trips, and the P V
+                // that has to precede it is long done.  Measured: late wins at d = 128,
+                // early at d = 64.
+                const bool rescale = j > 0 && __any_sync(0xffffffffu, m_new > m);
+                float f = 1.0f;
+                if (rescale) {
                     FP8ATTN_STAMP(t * 8 + 7, j);
-                    if (!pv_done) {
-                        w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
-                        tc_fence_after_sync();
-                        pv_done = true;
-                    }
-                    // the maximum moved for some row of this warp: rescale O and l
-                    const float f = ex2((m - m_new) * c);
+                    f = ex2((m - m_new) * c);
                     const uint64_t ff = pack2(f, f);
                     l2a = mul2(l2a, ff);
                     l2b = mul2(l2b, ff);
+                    if (!C::kLateRescale) {
+                        if (!pv_done) {
+                            w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                            tc_fence_after_sync();
+                            pv_done = true;
+                        }
 #pragma unroll
-                    for (int q = 0; q < kD / 16; ++q) {
-                        uint32_t o[16];
-                        tmem_ld_x16(tO + q * 16, o);
-                        tmem_wait_ld_x16(o);
+                        for (int q = 0; q < kD / 16; ++q) {
+                            uint32_t o[16];
+                            tmem_ld_x16(tO + q * 16, o);
+                            tmem_wait_ld_x16(o);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                        tmem_st_x16(tO + q * 16, o);
+                            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                            tmem_st_x16(tO + q * 16, o);
+                        }
                     }
                 }
                 m = m_new;
@@ -623,6 +633,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         FP8ATTN_STAMP(t * 8 + 5, j);
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
+                        pv_done = true;
                         FP8ATTN_STAMP(t * 8 + 6, j);
                     }
                     tmem_st_cols<kPPer32>(tP + (uint32_t)((C::kPBufs == 2 ? (j & 1) * C::kPCols : 0) + (k0 / 32) * kPPer32), p);
@@ -633,6 +644,24 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     // has, the buffer that the NEXT step writes (the one it read) is free.
                     // That write comes after the next step's fence behind its wait for S.
                     w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                    pv_done = true;
+                    if (C::kLateRescale && rescale) tc_fence_after_sync();
+                }
+                if (C::kLateRescale && rescale) {
+                    if (!pv_done) {
+                        w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
+                        tc_fence_after_sync();
+                    }
+#pragma unroll
+                    for (int q = 0; q < kD / 64; ++q) {
+                        uint32_t o[64];
+                        tmem_ld_cols<64>(tO + q * 64, o);
+                        tmem_wait_ld_cols<64>(o);
+#pragma unroll
+                        for (int i = 0; i < 64; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st_x32(tO + q * 64, o);
+                        tmem_st_x32(tO + q * 64 + 32, o + 32);
+                    }
                 }
                 tmem_wait_st();
                 tc_fence_before_sync();
