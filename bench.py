@@ -29,7 +29,7 @@ sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from an ncu capture of the
 # same workload (summaries under profiles/); None where no capture exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"C3": 219.7e6 + 138.0e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"C3": 219.0e6 + 136.6e6}
 NOMINAL_FP8_OVER_BF16 = 2.0           # dense tensor peak ratio (4.5 / 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
