@@ -87,6 +87,44 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(self.sm)}
 
 
+def library_fp8_gemm_rate(seconds: float = 3.0, n: int = 8192):
+    """Dense e4m3 GEMM rate of the vendor library on this GPU (TFLOP/s): best of 10 single
+    calls and back-to-back calls for `seconds` under the power cap.  Context for the roofline
+    only (what the tensor cores sustain on FP8 operands here); nothing on the timed path."""
+    import time
+    import torch
+    a = (torch.randn(n, n, device="cuda") * 0.5).to(torch.float8_e4m3fn)
+    b = (torch.randn(n, n, device="cuda") * 0.5).to(torch.float8_e4m3fn).t()
+    one = torch.tensor(1.0, device="cuda")
+
+    def gemm():
+        return torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+
+    for _ in range(3):
+        gemm()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        gemm()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    calls, t0 = 0, time.time()
+    e0.record()
+    while time.time() - t0 < seconds:
+        for _ in range(50):
+            gemm()
+        calls += 50
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    flop = 2.0 * n ** 3
+    return flop / best / 1e9, flop * calls / e0.elapsed_time(e1) / 1e9
+
+
 def oracle_sample(w, rows_per_head: int, seed: int = 0):
     """Time the CPU oracle, as it stands, on a bounded sample of workload ``w``:
     the full per-head quantization of K, V and both query tensors, then exact
@@ -160,6 +198,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=96, help="oracle sample: query rows per head and call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-bf16", action="store_true")
+    ap.add_argument("--no-fp8-gemm", action="store_true", help="skip the library FP8 GEMM rate (context figure)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -367,6 +406,13 @@ def main():
         cpu_baseline = {"value": v, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
                         "sample": info["sample"]}
 
+    fp8_gemm = None
+    if rank == 0 and world == 1 and not args.no_fp8_gemm:
+        try:
+            fp8_gemm = library_fp8_gemm_rate()
+        except Exception as e:      # context figure only: report why it is missing
+            fp8_gemm = str(e)[:120]
+
     if rank == 0:
         flops = w.flops
         tf_step = world * flops / (ms_step * 1e-3) / 1e12
@@ -392,7 +438,13 @@ def main():
                          "frac": tf_attn / peak_fp8, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
                          "peak_source": f"2 x bf16_tflops_sustained ({peak_kind}), nominal fp8:bf16 ratio",
                          "frac_of_burst_peak": tf_attn / peak_fp8_burst,
-                         "frac_of_nominal_4500": tf_attn / 4500.0},
+                         "frac_of_nominal_4500": tf_attn / 4500.0,
+                         "library_fp8_gemm_tflops": None if not isinstance(fp8_gemm, tuple) else
+                         {"burst": fp8_gemm[0], "sustained": fp8_gemm[1],
+                          "how": "torch._scaled_mm e4m3 8192^3, best of 10 / back to back for 3 s, same run"},
+                         "frac_of_library_fp8_gemm_sustained": None if not isinstance(fp8_gemm, tuple)
+                         else tf_attn / fp8_gemm[1],
+                         "library_fp8_gemm_error": fp8_gemm if isinstance(fp8_gemm, str) else None},
             "cpu_baseline": cpu_baseline,
             "breakdown": {
                 "ms_quantize": ms_quant, "ms_attention_fp8": ms_attn, "ms_attention_bf16": ms_bf16,
