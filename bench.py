@@ -163,6 +163,10 @@ def oracle_sample(w, rows_per_head: int, seed: int = 0):
     return flops / seconds / 1e12, info
 
 
+def workload_label(w) -> str:
+    return f"{w.name}: B={w.B} H={w.H} d={w.d} n_train={w.n_train} n_test={w.n_test}"
+
+
 def run_reference(args, w):
     """--impl reference: the CPU oracle, timed on the host cores, rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
@@ -180,8 +184,9 @@ def run_reference(args, w):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * sec, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "n_train": w.n_train,
-                   "n_test": w.n_test},
+        "config": {"workload": workload_label(w),
+                   "step": "oracle quantize + exact attention over the dequantized operands, "
+                           "a bounded sample of the step's rows"},
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
                          "sample": info["sample"]},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -425,7 +430,7 @@ def main():
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
             "data": "synthetic",
-            "config": {"workload": f"{w.name}: B={w.B} H={w.H} d={w.d} n_train={w.n_train} n_test={w.n_test}",
+            "config": {"workload": workload_label(w),
                        "step": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward",
                        "l2": "inputs larger than L2 (bf16 inputs %.0f MB)" % (h2d / 1e6),
                        "replicas": world},
