@@ -65,6 +65,15 @@ int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d,
                      const float* scale_in, void* x_fp8, float* scale_out,
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* fp8attn_quantize with a flags word.  FP8ATTN_INPUT_FP16: x holds IEEE fp16
+ * instead of bf16 (the paper's kernel benchmark table runs in float16); the
+ * arithmetic is the same, on the exact fp32 value of each input.  flags = 0 is
+ * fp8attn_quantize.  Unknown flag bits return FP8ATTN_ERR_INVALID_ARG. */
+#define FP8ATTN_INPUT_FP16 2u
+int fp8attn_quantize_ex(const void* x_16bit, int B, int H, int64_t rows, int d,
+                        const float* scale_in, void* x_fp8, float* scale_out, uint32_t flags,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The four quantizations of one ICL attention call in two launches instead of
  * seven (same arithmetic and bit-identical results to four fp8attn_quantize
  * calls): per-head absmax scales for Q_train, K and V (paper Eq. 2), and Q_test
@@ -89,7 +98,8 @@ int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, cons
  * dynamic scales).  Test predictions then depend on the test batch.  Without
  * the flag the scale comes from the train queries alone (the paper's proposal).
  * The "per-call query scale" ablation arm needs no flag: quantize the test
- * queries with fp8attn_quantize and scale_in = NULL. */
+ * queries with fp8attn_quantize and scale_in = NULL.
+ * FP8ATTN_INPUT_FP16 (above): all four inputs are IEEE fp16. */
 #define FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS 1u
 int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test,
                             int B, int H, int64_t n_train, int64_t n_test, int d,
@@ -143,9 +153,26 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
  * query scale stays head h's train-query scale).  Train rows are unaffected.
  * K and V are still passed, and were quantized, as full [B,H,n_train,d] tensors,
  * so both attention calls consume the same quantized K/V entries.
+ *
+ * FP8ATTN_TEST_ROWS_ONLY runs the test->train call alone: only out_test is
+ * written, q_train and out_train are not read or written and may be NULL, and
+ * n_test must be >= 1.  Together with the plain call at n_test = 0 (the
+ * train->train call alone) this gives the arms of the paper's precision
+ * ablation (results section, table of quantization arms: FP8 in the train
+ * context only, in the test context only, in both): run one call through
+ * fp8attn_icl_forward_ex and the other through bf16attn_icl_forward_ex.  The
+ * test rows' results are bit-identical to those of the combined call.
+ *
+ * FP8ATTN_IO_FP16 switches the 16-bit tensors of the call from bf16 to IEEE
+ * fp16 (the paper's kernel benchmark table runs in float16): the outputs of
+ * fp8attn_icl_forward_ex, and the inputs, the on-chip probabilities and the
+ * outputs of bf16attn_icl_forward_ex (which then is an fp16 kernel).
+ *
  * Unknown flag bits return FP8ATTN_ERR_INVALID_ARG.  flags = 0 is the plain call.
  */
 #define FP8ATTN_TEST_ROWS_USE_KV_HEAD0 1u
+#define FP8ATTN_TEST_ROWS_ONLY 2u
+#define FP8ATTN_IO_FP16 4u
 int fp8attn_icl_forward_ex(const void* q_train_fp8, const void* q_test_fp8,
                            const void* k_fp8, const void* v_fp8,
                            const float* scale_q, const float* scale_k, const float* scale_v,

@@ -70,6 +70,13 @@ def _load():
                 ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
                 ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                 ctypes.c_int]
+            lib.oracle_quantize_ex.restype = None
+            lib.oracle_quantize_ex.argtypes = [
+                ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+                ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                ctypes.c_int]
+            lib.oracle_half_to_float.restype = ctypes.c_float
+            lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
             lib.oracle_icl_attention_rows.restype = None
             lib.oracle_icl_attention_rows.argtypes = [ctypes.POINTER(_AttnArgs)]
             lib.oracle_perturb.restype = None
@@ -121,9 +128,18 @@ def e4m3_decode_table() -> np.ndarray:
 
 # ---- quantize (Eq. 2) --------------------------------------------------------
 
+_DTYPE16 = {"bf16": 0, "fp16": 1}
+
+
+def half_to_float(bits: int) -> float:
+    """Value of one IEEE fp16 bit pattern, by the format's definition."""
+    return float(_load().oracle_half_to_float(int(bits) & 0xFFFF))
+
+
 def quantize(x_bf16_bits: np.ndarray, scale_in: np.ndarray | None = None,
-             nthreads: int | None = None):
-    """bf16 bits [B,H,R,d] -> (codes uint8 [B,H,R,d], scale fp32 [B,H])."""
+             nthreads: int | None = None, dtype16: str = "bf16"):
+    """16-bit patterns [B,H,R,d] (bf16, or IEEE fp16 with dtype16="fp16")
+    -> (codes uint8 [B,H,R,d], scale fp32 [B,H])."""
     x = np.ascontiguousarray(x_bf16_bits, dtype=np.uint16)
     B, H, R, d = x.shape
     codes = np.empty(x.shape, dtype=np.uint8)
@@ -132,8 +148,8 @@ def quantize(x_bf16_bits: np.ndarray, scale_in: np.ndarray | None = None,
     if scale_in is not None:
         s_in = np.ascontiguousarray(scale_in, dtype=np.float32).reshape(B, H)
     nt = nthreads or hardware_threads()
-    _load().oracle_quantize(_ptr(x), B, H, R, d, _ptr(s_in), _ptr(codes),
-                            _ptr(scale), nt)
+    _load().oracle_quantize_ex(_ptr(x), _DTYPE16[dtype16], B, H, R, d, _ptr(s_in), _ptr(codes),
+                               _ptr(scale), nt)
     return codes, scale
 
 
@@ -141,11 +157,12 @@ def quantize(x_bf16_bits: np.ndarray, scale_in: np.ndarray | None = None,
 
 def icl_attention_rows(q, k, v, rows, *, sq=None, sk=None, sv=None,
                        alpha: float | None = None, mode: str = "exact",
-                       nthreads: int | None = None):
+                       nthreads: int | None = None, dtype16: str = "bf16"):
     """Attention outputs of selected query rows against ALL train keys.
 
     q: [B,H,nq,d], k/v: [B,H,N,d]; uint8 = FP8 codes (scales [B,H] required),
-    uint16 = bf16 bits (no scales).  ``rows``: 1-D int array of query rows,
+    uint16 = bf16 bits, or IEEE fp16 bits with dtype16="fp16" (no scales).
+    ``rows``: 1-D int array of query rows,
     evaluated for every (b,h).  mode "exact": returns (A, Abs, Bnd) fp64
     [B,H,len(rows),d]; mode "p8": returns the two-pass e4m3-P result (A only,
     bf16-rounded values held in fp64).
@@ -175,7 +192,8 @@ def icl_attention_rows(q, k, v, rows, *, sq=None, sk=None, sv=None,
     Abs = np.zeros(shape, dtype=np.float64)
     Bnd = np.zeros(shape, dtype=np.float64)
     args = _AttnArgs(
-        q=_ptr(q), k=_ptr(k), v=_ptr(v), is_fp8=int(is_fp8),
+        q=_ptr(q), k=_ptr(k), v=_ptr(v),
+        is_fp8=1 if is_fp8 else (2 if _DTYPE16[dtype16] else 0),
         sq=_ptr(scales[0]), sk=_ptr(scales[1]), sv=_ptr(scales[2]),
         B=B, H=H, nq=nq, n_train=N, d=d, alpha=float(alpha),
         rows=_ptr(rows), n_rows=rows.size, mode={"exact": 0, "p8": 1}[mode],

@@ -11,6 +11,9 @@
 // s = amax/448 and the quotient x/s of the quantizer (Eq. 2), which are IEEE
 // fp32 operations because their rounding decides the FP8 code.
 //
+// 16-bit inputs are bf16 or, where a dtype16 argument says so, IEEE fp16; both
+// are read by the format's definition.
+//
 // Parity pins: every function below is pinned by tests/test_oracle_*.py against
 // facts that do not come from this file (format definition, closed forms,
 // numpy fp64 brute force, a third-party FP8 cast, values the paper prints).
@@ -89,6 +92,22 @@ float bf16_to_float(uint16_t b) {
     return f;
 }
 
+// IEEE binary16 by definition: 1 sign, 5 exponent bits (bias 15), 10 mantissa bits;
+// exponent 0 holds zero and the subnormals k * 2^-24, exponent 31 infinity and NaN.
+float half_to_float(uint16_t h) {
+    const int sign = (h >> 15) & 1, e = (h >> 10) & 0x1F, m = h & 0x3FF;
+    double v;
+    if (e == 0) v = std::ldexp((double)m, -24);
+    else if (e == 31) v = m ? std::nan("") : INFINITY;
+    else v = std::ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
+}
+
+// One 16-bit input element as fp32: dtype16 0 = bf16, 1 = IEEE fp16.
+static inline float in16_to_float(uint16_t b, int dtype16) {
+    return dtype16 ? half_to_float(b) : bf16_to_float(b);
+}
+
 // Round an fp32 value to the nearest bf16 (ties to even), returned as float.
 float round_to_bf16(float x) {
     uint32_t u;
@@ -150,16 +169,19 @@ void oracle_e4m3_encode_array(const float* y, int64_t n, uint8_t* out) {
     for (int64_t i = 0; i < n; ++i) out[i] = encode((double)y[i]);
 }
 
+float oracle_half_to_float(uint16_t h) { return half_to_float(h); }
+
 // ---- quantize (Eq. 2) ------------------------------------------------------
-// x: bf16 bit patterns [B,H,R,d] contiguous.  scale_in: NULL or [B*H] fp32.
+// x: bf16 (dtype16 = 0) or IEEE fp16 (dtype16 = 1) bit patterns [B,H,R,d] contiguous.
+// scale_in: NULL or [B*H] fp32.
 // codes: [B,H,R,d] bytes.  scale_out: [B*H] fp32 (may be NULL).
 // Per (b,h): amax = max|x|; s = amax/448 in fp32 (s = 1 for an all-zero head);
 // with scale_in the given scale is used instead (shared train-query scale).
 // Per entry: y = x/s in fp32, clamp to [-448,448], round to nearest e4m3,
 // ties to even.
-void oracle_quantize(const uint16_t* x, int B, int H, int64_t R, int d,
-                     const float* scale_in, uint8_t* codes, float* scale_out,
-                     int nthreads) {
+void oracle_quantize_ex(const uint16_t* x, int dtype16, int B, int H, int64_t R, int d,
+                        const float* scale_in, uint8_t* codes, float* scale_out,
+                        int nthreads) {
     int64_t per_head = R * (int64_t)d;
     parallel_for((int64_t)B * H, nthreads, [&](int64_t bh) {
         const uint16_t* xs = x + bh * per_head;
@@ -170,19 +192,25 @@ void oracle_quantize(const uint16_t* x, int B, int H, int64_t R, int d,
         } else {
             float amax = 0.0f;
             for (int64_t i = 0; i < per_head; ++i) {
-                float a = std::fabs(bf16_to_float(xs[i]));
+                float a = std::fabs(in16_to_float(xs[i], dtype16));
                 if (a > amax) amax = a;
             }
             s = (amax == 0.0f) ? 1.0f : amax / 448.0f;  // IEEE fp32 divide
         }
         if (scale_out) scale_out[bh] = s;
         for (int64_t i = 0; i < per_head; ++i) {
-            float yc = bf16_to_float(xs[i]) / s;  // IEEE fp32 divide
+            float yc = in16_to_float(xs[i], dtype16) / s;  // IEEE fp32 divide
             if (yc > 448.0f) yc = 448.0f;
             if (yc < -448.0f) yc = -448.0f;
             cs[i] = encode((double)yc);
         }
     });
+}
+
+void oracle_quantize(const uint16_t* x, int B, int H, int64_t R, int d,
+                     const float* scale_in, uint8_t* codes, float* scale_out,
+                     int nthreads) {
+    oracle_quantize_ex(x, 0, B, H, R, d, scale_in, codes, scale_out, nthreads);
 }
 
 // ---- attention over dequantized operands (Eq. 1, two-call ICL structure) ---
@@ -192,8 +220,8 @@ void oracle_quantize(const uint16_t* x, int B, int H, int64_t R, int d,
 // held as fp64, j running over the n_train key/value rows of head (b,h) ONLY:
 // train queries and test queries both attend to train rows, never to test rows.
 //
-// Inputs are either FP8 codes (is_fp8=1: uint8, decoded by table) or bf16 bit
-// patterns (is_fp8=0: uint16, scales must be 1), so the same routine is the
+// Inputs are either FP8 codes (is_fp8=1: uint8, decoded by table) or 16-bit
+// patterns (is_fp8=0: bf16, is_fp8=2: IEEE fp16; scales must be 1), so the same routine is the
 // reference for the quantized path and for the 16-bit comparison path.
 //
 // rows: n_rows query-row indices (into the nq rows of q) evaluated for every
@@ -221,8 +249,8 @@ struct AttnArgs {
 };
 
 static double load_elem(const void* p, int is_fp8, int64_t idx) {
-    if (is_fp8) return decode(((const uint8_t*)p)[idx]);
-    return (double)bf16_to_float(((const uint16_t*)p)[idx]);
+    if (is_fp8 == 1) return decode(((const uint8_t*)p)[idx]);
+    return (double)in16_to_float(((const uint16_t*)p)[idx], is_fp8 == 2);
 }
 
 void oracle_icl_attention_rows(const AttnArgs* a_) {

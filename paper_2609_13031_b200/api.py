@@ -24,10 +24,15 @@ EXPORTS = (
     "fp8attn_launch_count", "fp8attn_quantize_noalloc",
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
     "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex", "fp8attn_perturb",
-    "fp8attn_selftest_wait_timeout",
+    "fp8attn_selftest_wait_timeout", "fp8attn_quantize_ex",
 )
+# flags of fp8attn_quantize_ex / fp8attn_quantize_qkv_ex
 QUERY_SCALE_FROM_ALL_ROWS = 1
+INPUT_FP16 = 2
+# flags of fp8attn_icl_forward_ex / bf16attn_icl_forward_ex
 TEST_ROWS_USE_KV_HEAD0 = 1
+TEST_ROWS_ONLY = 2
+IO_FP16 = 4
 GATE_TRAIN_ROWS = 8192
 
 _lib = None
@@ -54,6 +59,8 @@ def load() -> ctypes.CDLL:
                              ctypes.c_size_t)
     lib.fp8attn_quantize.restype = i32
     lib.fp8attn_quantize.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp, sz, vp]
+    lib.fp8attn_quantize_ex.restype = i32
+    lib.fp8attn_quantize_ex.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, ctypes.c_uint32, vp, sz, vp]
     lib.fp8attn_quantize_noalloc.restype = i32
     lib.fp8attn_quantize_noalloc.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp]
     lib.fp8attn_icl_forward.restype = i32
@@ -128,17 +135,28 @@ def _dims(x: torch.Tensor):
     return x.shape
 
 
+def _is16(t: torch.Tensor) -> bool:
+    return t.dtype in (torch.bfloat16, torch.float16)
+
+
 def quantize(x: torch.Tensor, workspace: torch.Tensor, scale_in: torch.Tensor | None = None,
              out: torch.Tensor | None = None, scale_out: torch.Tensor | None = None):
-    """fp8attn_quantize: bf16 [B,H,rows,d] -> (e4m3 codes as uint8 [B,H,rows,d], fp32 scale [B,H])."""
+    """fp8attn_quantize (bf16 input) / fp8attn_quantize_ex with FP8ATTN_INPUT_FP16 (fp16 input):
+    [B,H,rows,d] -> (e4m3 codes as uint8 [B,H,rows,d], fp32 scale [B,H])."""
     B, H, rows, d = _dims(x)
-    assert x.dtype == torch.bfloat16
+    assert _is16(x)
     if out is None:
         out = torch.empty((B, H, rows, d), dtype=torch.uint8, device=x.device)
     if scale_out is None:
         scale_out = torch.empty((B, H), dtype=torch.float32, device=x.device)
     if scale_in is not None:
         assert scale_in.dtype == torch.float32 and scale_in.is_contiguous() and scale_in.numel() == B * H
+    if x.dtype == torch.float16:
+        rc = load().fp8attn_quantize_ex(_ptr(x), B, H, rows, d, _ptr(scale_in), _ptr(out),
+                                        _ptr(scale_out), INPUT_FP16, _ptr(workspace),
+                                        workspace.numel(), _stream())
+        _check("fp8attn_quantize_ex", rc)
+        return out, scale_out
     rc = load().fp8attn_quantize(_ptr(x), B, H, rows, d, _ptr(scale_in), _ptr(out), _ptr(scale_out),
                                  _ptr(workspace), workspace.numel(), _stream())
     _check("fp8attn_quantize", rc)
@@ -168,6 +186,10 @@ def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
     dev = k.device
+    for t in (q_train, k, v) + (() if q_test is None else (q_test,)):
+        assert t.dtype == k.dtype and _is16(t)
+    if k.dtype == torch.float16:
+        flags |= INPUT_FP16
     o = dict(out or {})
     for name, rows in (("q8", n_train), ("k8", n_train), ("v8", n_train), ("t8", n_test)):
         if name not in o:
@@ -214,17 +236,29 @@ def gate_use_fp8(n_train: int) -> bool:
 
 
 def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
-                    softmax_scale: float = 0.0, out_train=None, out_test=None, flags: int = 0):
+                    softmax_scale: float = 0.0, out_train=None, out_test=None, flags: int = 0,
+                    out_dtype=torch.bfloat16):
     """fp8attn_icl_forward (flags == 0) / fp8attn_icl_forward_ex on uint8 e4m3
-    tensors; returns (out_train, out_test) bf16."""
+    tensors; returns (out_train, out_test) in ``out_dtype`` (bf16, or fp16 =
+    FP8ATTN_IO_FP16).  With TEST_ROWS_ONLY ``q_train`` may be None and out_train
+    is None."""
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
-    for t in (q_train, k, v):
+    test_only = bool(flags & TEST_ROWS_ONLY)
+    for t in (k, v) + (() if test_only else (q_train,)):
         assert t.dtype == torch.uint8
-    if out_train is None:
-        out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
+    for t in (out_train, out_test):
+        if t is not None:
+            out_dtype = t.dtype
+    assert out_dtype in (torch.bfloat16, torch.float16)
+    if out_dtype == torch.float16:
+        flags |= IO_FP16
+    if out_train is None and not test_only:
+        out_train = torch.empty((B, H, n_train, d), dtype=out_dtype, device=k.device)
     if out_test is None and n_test > 0:
-        out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+        out_test = torch.empty((B, H, n_test, d), dtype=out_dtype, device=k.device)
+    if test_only:
+        q_train, out_train = None, None
     if flags:
         rc = load().fp8attn_icl_forward_ex(
             _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v),
@@ -244,15 +278,25 @@ def icl_forward_fp8(q_train, q_test, k, v, scale_q, scale_k, scale_v, workspace,
 
 def icl_forward_bf16(q_train, q_test, k, v, workspace, softmax_scale: float = 0.0,
                      out_train=None, out_test=None, flags: int = 0):
-    """bf16attn_icl_forward on bf16 tensors; returns (out_train, out_test) bf16."""
+    """bf16attn_icl_forward on bf16 tensors (or, with fp16 tensors, its
+    FP8ATTN_IO_FP16 form); returns (out_train, out_test) in the input dtype.
+    With TEST_ROWS_ONLY ``q_train`` may be None and out_train is None."""
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
-    for t in (q_train, k, v):
-        assert t.dtype == torch.bfloat16
-    if out_train is None:
-        out_train = torch.empty((B, H, n_train, d), dtype=torch.bfloat16, device=k.device)
+    test_only = bool(flags & TEST_ROWS_ONLY)
+    assert _is16(k)
+    for t in (v,) + (() if test_only else (q_train,)) + (() if q_test is None else (q_test,)):
+        assert t.dtype == k.dtype
+    if k.dtype == torch.float16:
+        flags |= IO_FP16
+    if out_train is None and not test_only:
+        out_train = torch.empty((B, H, n_train, d), dtype=k.dtype, device=k.device)
     if out_test is None and n_test > 0:
-        out_test = torch.empty((B, H, n_test, d), dtype=torch.bfloat16, device=k.device)
+        out_test = torch.empty((B, H, n_test, d), dtype=k.dtype, device=k.device)
+    for t in (out_train, out_test):
+        assert t is None or t.dtype == k.dtype
+    if test_only:
+        q_train, out_train = None, None
     if flags:
         rc = load().bf16attn_icl_forward_ex(
             _ptr(q_train), _ptr(q_test) if n_test else None, _ptr(k), _ptr(v), B, H, n_train, n_test,
@@ -285,7 +329,32 @@ def icl_attention(q_train, q_test, k, v, workspace=None, softmax_scale: float = 
     o = quantize_qkv(q_train, k, v, q_test if has_test else None, workspace)
     q8, k8, v8, sq, sk, sv = o["q8"], o["k8"], o["v8"], o["sq"], o["sk"], o["sv"]
     t8 = o["t8"] if has_test else None
-    return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale)
+    return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale, out_dtype=k.dtype)
+
+
+def icl_attention_arms(q_train, q_test, k, v, fp8_train: bool, fp8_test: bool, workspace=None,
+                       softmax_scale: float = 0.0):
+    """The arms of the paper's precision ablation: the train->train call and the
+    test->train call each run either in FP8 or in 16 bits (n_test = 0 and
+    TEST_ROWS_ONLY select one call).  Returns (out_train, out_test)."""
+    B, H, _, _ = _dims(k)
+    if workspace is None:
+        workspace = new_workspace(B, H, k.device)
+    assert q_test is not None and q_test.shape[2] > 0
+    if fp8_train == fp8_test:
+        if fp8_train:
+            return icl_attention(q_train, q_test, k, v, workspace, softmax_scale)
+        return icl_forward_bf16(q_train, q_test, k, v, workspace, softmax_scale)
+    o = quantize_qkv(q_train, k, v, q_test, workspace)
+    fp8 = (o["q8"], o["t8"], o["k8"], o["v8"], o["sq"], o["sk"], o["sv"])
+    if fp8_train:
+        out_train, _ = icl_forward_fp8(fp8[0], None, *fp8[2:], workspace, softmax_scale, out_dtype=k.dtype)
+        _, out_test = icl_forward_bf16(None, q_test, k, v, workspace, softmax_scale, flags=TEST_ROWS_ONLY)
+    else:
+        out_train, _ = icl_forward_bf16(q_train, None, k, v, workspace, softmax_scale)
+        _, out_test = icl_forward_fp8(None, fp8[1], *fp8[2:], workspace, softmax_scale,
+                                      flags=TEST_ROWS_ONLY, out_dtype=k.dtype)
+    return out_train, out_test
 
 
 def icl_attention_gated(q_train, q_test, k, v, workspace=None, softmax_scale: float = 0.0):

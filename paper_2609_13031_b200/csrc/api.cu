@@ -41,14 +41,18 @@ int forward(bool fp8, const void* q_train, const void* q_test, const void* k, co
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0 || n_train > 0x7fffff00ll || n_test > 0x7fffff00ll)
         return FP8ATTN_ERR_INVALID_ARG;
-    if (!q_train || !k || !v || !out_train) return FP8ATTN_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(FP8ATTN_TEST_ROWS_USE_KV_HEAD0 | FP8ATTN_TEST_ROWS_ONLY | FP8ATTN_IO_FP16))
+        return FP8ATTN_ERR_INVALID_ARG;
+    const bool test_only = (flags & FP8ATTN_TEST_ROWS_ONLY) != 0;
+    if (test_only && n_test < 1) return FP8ATTN_ERR_INVALID_ARG;
+    if (!k || !v || (!test_only && (!q_train || !out_train))) return FP8ATTN_ERR_INVALID_ARG;
     if (n_test > 0 && (!q_test || !out_test)) return FP8ATTN_ERR_INVALID_ARG;
     if (fp8 && (!sq || !sk || !sv)) return FP8ATTN_ERR_INVALID_ARG;
-    if (!aligned(q_train, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out_train, 16) ||
+    if (!aligned(k, 16) || !aligned(v, 16) ||
+        (!test_only && (!aligned(q_train, 16) || !aligned(out_train, 16))) ||
         (n_test > 0 && (!aligned(q_test, 16) || !aligned(out_test, 16))))
         return FP8ATTN_ERR_INVALID_ARG;
     if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return FP8ATTN_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)FP8ATTN_TEST_ROWS_USE_KV_HEAD0) return FP8ATTN_ERR_INVALID_ARG;
     rc = check_workspace(workspace, workspace_bytes_, B, H);
     if (rc != FP8ATTN_OK) return rc;
     rc = check_device();
@@ -74,8 +78,16 @@ extern "C" {
 int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d, const float* scale_in,
                      void* x_fp8, float* scale_out, void* workspace, size_t workspace_bytes_,
                      void* cuda_stream) {
+    return fp8attn_quantize_ex(x_bf16, B, H, rows, d, scale_in, x_fp8, scale_out, 0u, workspace,
+                               workspace_bytes_, cuda_stream);
+}
+
+int fp8attn_quantize_ex(const void* x_bf16, int B, int H, int64_t rows, int d, const float* scale_in,
+                        void* x_fp8, float* scale_out, uint32_t flags, void* workspace,
+                        size_t workspace_bytes_, void* cuda_stream) {
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
+    if (flags & ~(uint32_t)FP8ATTN_INPUT_FP16) return FP8ATTN_ERR_INVALID_ARG;
     if (rows < 0) return FP8ATTN_ERR_INVALID_ARG;
     if (rows > 0 && (!x_bf16 || !x_fp8)) return FP8ATTN_ERR_INVALID_ARG;
     if (!scale_in && !scale_out) return FP8ATTN_ERR_INVALID_ARG;
@@ -87,7 +99,7 @@ int fp8attn_quantize(const void* x_bf16, int B, int H, int64_t rows, int d, cons
     if (rc != FP8ATTN_OK) return rc;
     uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
     return launch_quantize(x_bf16, (int64_t)B * H, rows * (int64_t)d, scale_in, x_fp8, scale_out, amax,
-                           static_cast<cudaStream_t>(cuda_stream));
+                           flags, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test, int B,
@@ -97,7 +109,8 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS) return FP8ATTN_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS | FP8ATTN_INPUT_FP16))
+        return FP8ATTN_ERR_INVALID_ARG;
     if (!q_train || !k || !v || !q_train_fp8 || !k_fp8 || !v_fp8 || !scale_q || !scale_k || !scale_v)
         return FP8ATTN_ERR_INVALID_ARG;
     if (n_test > 0 && (!q_test || !q_test_fp8)) return FP8ATTN_ERR_INVALID_ARG;

@@ -54,7 +54,9 @@ enum : uint32_t {
     kWaitSFree, kWaitPFree, kWaitSelfTest
 };
 
-template <bool kFp8, int kD>
+// kFp8: e4m3 operands and P (else 16-bit operands and P).  kHalf: the 16-bit type of the
+// 16-bit kernel is IEEE fp16 instead of bf16 (ignored when kFp8).
+template <bool kFp8, int kD, bool kHalf = false>
 struct Cfg {
     static constexpr int kES = kFp8 ? 1 : 2;                    // element bytes
     static constexpr int kRowBytes = kD * kES;
@@ -68,7 +70,7 @@ struct Cfg {
     static constexpr int kUmmaK = 32 / kES;                     // elements per MMA K step
     static constexpr int kStages = kKVTileBytes >= 32768 ? 2 : 4;  // K ring and V ring depth
     static constexpr uint32_t kSwizzle = kBoxBytes == 128 ? kSwizzle128 : kSwizzle64;
-    static constexpr uint32_t kFmt = kFp8 ? 0u : 1u;            // e4m3 / bf16
+    static constexpr uint32_t kFmt = (kFp8 || kHalf) ? 0u : 1u; // e4m3 (kind::f8f6f4); f16 / bf16 (kind::f16)
     static constexpr uint32_t kIdescQK = idesc(kFmt, kFmt, false, false, kTileM, kKeys);
     static constexpr uint32_t kIdescPV = idesc(kFmt, kFmt, false, true, kTileM, kD);
     static constexpr int kPCols = kKeys * kES / 4;              // TMEM columns of a P tile
@@ -156,6 +158,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two fp32 -> two 16-bit values of the call's 16-bit type (bf16, or IEEE fp16)
+template <bool kHalf>
+__device__ __forceinline__ uint32_t pack_16x2(float lo, float hi) {
+    return kHalf ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
 }
 
 // ---- packed fp32x2 arithmetic (two lanes per instruction on sm_100) ----
@@ -303,17 +315,18 @@ struct KernelArgs {
     int blocks_train, blocks_test;   // 256-row query blocks per head
     int heads;                       // H, to find head 0 of a table
     int test_kv_head0;               // test rows read K, V and their scales from head 0 of their table
+    int out_half;                    // FP8 kernel: outputs are IEEE fp16 instead of bf16
     float softmax_scale;
     uint32_t* status;
 };
 
-template <bool kFp8, int kD>
+template <bool kFp8, int kD, bool kHalf>
 __global__ void __launch_bounds__(kNumThreads, 1)
 icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                      const __grid_constant__ CUtensorMap map_q_test,
                      const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const KernelArgs args) {
-    using C = Cfg<kFp8, kD>;
+    using C = Cfg<kFp8, kD, kHalf>;
     constexpr int kKeys = C::kKeys;
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
@@ -625,8 +638,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         if (kFp8) {
                             p[i / 4] = pack_e4m3x4(p0, p1, p2, p3);
                         } else {
-                            p[i / 2] = pack_bf16x2(p0, p1);
-                            p[i / 2 + 1] = pack_bf16x2(p2, p3);
+                            p[i / 2] = pack_16x2<kHalf>(p0, p1);
+                            p[i / 2 + 1] = pack_16x2<kHalf>(p2, p3);
                         }
                     }
                     if (C::kPBufs == 1 && k0 == 0 && !pv_done) {
@@ -681,6 +694,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             tc_fence_after_sync();
             const int64_t row = row0 + t * kTileM + row_in_tile;
             const float inv = sv_scale / l;
+            const bool out_half = kFp8 ? args.out_half != 0 : kHalf;   // 16-bit type of the outputs
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
                                  ((int64_t)bh * q_rows + row) * kD;
 #pragma unroll
@@ -692,10 +706,18 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
                         uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-                        v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-                        v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-                        v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                        auto val = [&](int k) { return __uint_as_float(o[i + k]) * inv; };
+                        if (out_half) {
+                            v.x = pack_f16x2(val(0), val(1));
+                            v.y = pack_f16x2(val(2), val(3));
+                            v.z = pack_f16x2(val(4), val(5));
+                            v.w = pack_f16x2(val(6), val(7));
+                        } else {
+                            v.x = pack_bf16x2(val(0), val(1));
+                            v.y = pack_bf16x2(val(2), val(3));
+                            v.z = pack_bf16x2(val(4), val(5));
+                            v.w = pack_bf16x2(val(6), val(7));
+                        }
                         *reinterpret_cast<uint4*>(out + q * 32 + i) = v;
                     }
                 }
@@ -708,14 +730,17 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <bool kFp8, int kD>
+template <bool kFp8, int kD, bool kHalf>
 int launch(const AttnParams& p, cudaStream_t stream) {
-    using C = Cfg<kFp8, kD>;
+    using C = Cfg<kFp8, kD, kHalf>;
     const int64_t heads = (int64_t)p.B * p.H;
+    const bool test_only = (p.flags & FP8ATTN_TEST_ROWS_ONLY) != 0;
     CUtensorMap mq_train, mq_test, mk, mv;
-    if (!make_tensor_map(&mq_train, p.q_train, C::kES, heads, p.n_train, kD, kTileM, C::kBoxCols) ||
-        !make_tensor_map(&mk, p.k, C::kES, heads, p.n_train, kD, C::kKeys, C::kBoxCols) ||
+    if (!make_tensor_map(&mk, p.k, C::kES, heads, p.n_train, kD, C::kKeys, C::kBoxCols) ||
         !make_tensor_map(&mv, p.v, C::kES, heads, p.n_train, kD, C::kKeys, C::kBoxCols))
+        return FP8ATTN_ERR_CUDA;
+    if (!test_only &&
+        !make_tensor_map(&mq_train, p.q_train, C::kES, heads, p.n_train, kD, kTileM, C::kBoxCols))
         return FP8ATTN_ERR_CUDA;
     if (p.n_test > 0) {
         if (!make_tensor_map(&mq_test, p.q_test, C::kES, heads, p.n_test, kD, kTileM, C::kBoxCols))
@@ -723,19 +748,21 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     } else {
         mq_test = mq_train;
     }
+    if (test_only) mq_train = mq_test;   // never used: the work list has no train blocks
     KernelArgs a;
     a.scale_q = p.scale_q; a.scale_k = p.scale_k; a.scale_v = p.scale_v;
     a.out_train = p.out_train; a.out_test = p.out_test;
     a.n_train = p.n_train; a.n_test = p.n_test;
-    a.blocks_train = (int)((p.n_train + 2 * kTileM - 1) / (2 * kTileM));
+    a.blocks_train = test_only ? 0 : (int)((p.n_train + 2 * kTileM - 1) / (2 * kTileM));
     a.blocks_test = (int)((p.n_test + 2 * kTileM - 1) / (2 * kTileM));
     a.softmax_scale = p.softmax_scale;
     a.heads = p.H;
     a.test_kv_head0 = (p.flags & FP8ATTN_TEST_ROWS_USE_KV_HEAD0) ? 1 : 0;
+    a.out_half = (p.flags & FP8ATTN_IO_FP16) ? 1 : 0;
     a.status = p.status;
     const int64_t grid = heads * (a.blocks_train + a.blocks_test);
     if (grid > 0x7fffffffll) return FP8ATTN_ERR_UNSUPPORTED;
-    auto kern = icl_attention_kernel<kFp8, kD>;
+    auto kern = icl_attention_kernel<kFp8, kD, kHalf>;
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -780,8 +807,10 @@ int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream
 }
 
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {
-    if (fp8) return p.d == 64 ? launch<true, 64>(p, stream) : launch<true, 128>(p, stream);
-    return p.d == 64 ? launch<false, 64>(p, stream) : launch<false, 128>(p, stream);
+    if (fp8) return p.d == 64 ? launch<true, 64, false>(p, stream) : launch<true, 128, false>(p, stream);
+    if (p.flags & FP8ATTN_IO_FP16)
+        return p.d == 64 ? launch<false, 64, true>(p, stream) : launch<false, 128, true>(p, stream);
+    return p.d == 64 ? launch<false, 64, false>(p, stream) : launch<false, 128, false>(p, stream);
 }
 
 }  // namespace fp8attn

@@ -29,7 +29,7 @@ void count_launch();
 // quantize.cu
 int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
                     const float* scale_in, void* x_fp8, float* scale_out,
-                    uint32_t* amax_bits, cudaStream_t stream);
+                    uint32_t* amax_bits, uint32_t flags, cudaStream_t stream);
 
 int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,

@@ -1,4 +1,4 @@
-// Per-head absmax quantization of bf16 tensors to e4m3 (paper Eq. 2).
+// Per-head absmax quantization of bf16 (or IEEE fp16) tensors to e4m3 (paper Eq. 2).
 //
 // Two HBM-bound kernels per call:
 //   absmax_kernel    max |x| per head, packed bf16x2 max, one atomicMax per block
@@ -8,6 +8,7 @@
 // The conversion walks each head backwards so that it starts on the part of the
 // head the maximum pass touched last, which is still in L2.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <mutex>
 
@@ -25,36 +26,46 @@ __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
     return v;
 }
 
-__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) {
-    return *reinterpret_cast<__nv_bfloat162*>(&u);
-}
+// The two 16-bit input types: packed |x| / max for the reduction, and the exact
+// fp32 value of the low and high half of a 32-bit word for the conversion.
+template <bool kHalf> struct In16;
+template <> struct In16<false> {
+    using V2 = __nv_bfloat162;
+    static __device__ __forceinline__ V2 as2(uint32_t u) { return *reinterpret_cast<V2*>(&u); }
+    // an fp32 with the bf16 bits in its upper half is that value
+    static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+    static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+};
+template <> struct In16<true> {
+    using V2 = __half2;
+    static __device__ __forceinline__ V2 as2(uint32_t u) { return *reinterpret_cast<V2*>(&u); }
+    static __device__ __forceinline__ float lo(uint32_t w) { return __low2float(as2(w)); }
+    static __device__ __forceinline__ float hi(uint32_t w) { return __high2float(as2(w)); }
+};
 
 // One block's share of max |x| over head blockIdx.y (vecs_per_head 16-byte vectors),
 // merged into amax_bits[blockIdx.y].
+template <bool kHalf>
 __device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t vecs_per_head,
                                             uint32_t* __restrict__ amax_bits) {
+    using T = In16<kHalf>;
+    using V2 = typename T::V2;
+    auto am = [](uint32_t a, uint32_t b) { return __hmax2(__habs2(T::as2(a)), __habs2(T::as2(b))); };
     const uint4* xh = x + (int64_t)blockIdx.y * vecs_per_head;
-    __nv_bfloat162 m = as_bf162(0u);
+    V2 m = T::as2(0u);
     int64_t stride = (int64_t)gridDim.x * kThreads;
     int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     for (; i + 3 * stride < vecs_per_head; i += 4 * stride) {
         uint4 a = ld_nc_v4(xh + i), b = ld_nc_v4(xh + i + stride);
         uint4 c = ld_nc_v4(xh + i + 2 * stride), e = ld_nc_v4(xh + i + 3 * stride);
-        __nv_bfloat162 m0 = __hmax2(__habs2(as_bf162(a.x)), __habs2(as_bf162(a.y)));
-        __nv_bfloat162 m1 = __hmax2(__habs2(as_bf162(a.z)), __habs2(as_bf162(a.w)));
-        __nv_bfloat162 m2 = __hmax2(__habs2(as_bf162(b.x)), __habs2(as_bf162(b.y)));
-        __nv_bfloat162 m3 = __hmax2(__habs2(as_bf162(b.z)), __habs2(as_bf162(b.w)));
-        __nv_bfloat162 m4 = __hmax2(__habs2(as_bf162(c.x)), __habs2(as_bf162(c.y)));
-        __nv_bfloat162 m5 = __hmax2(__habs2(as_bf162(c.z)), __habs2(as_bf162(c.w)));
-        __nv_bfloat162 m6 = __hmax2(__habs2(as_bf162(e.x)), __habs2(as_bf162(e.y)));
-        __nv_bfloat162 m7 = __hmax2(__habs2(as_bf162(e.z)), __habs2(as_bf162(e.w)));
+        V2 m0 = am(a.x, a.y), m1 = am(a.z, a.w), m2 = am(b.x, b.y), m3 = am(b.z, b.w);
+        V2 m4 = am(c.x, c.y), m5 = am(c.z, c.w), m6 = am(e.x, e.y), m7 = am(e.z, e.w);
         m = __hmax2(m, __hmax2(__hmax2(__hmax2(m0, m1), __hmax2(m2, m3)),
                                __hmax2(__hmax2(m4, m5), __hmax2(m6, m7))));
     }
     for (; i < vecs_per_head; i += stride) {
         uint4 a = ld_nc_v4(xh + i);
-        m = __hmax2(m, __hmax2(__hmax2(__habs2(as_bf162(a.x)), __habs2(as_bf162(a.y))),
-                               __hmax2(__habs2(as_bf162(a.z)), __habs2(as_bf162(a.w)))));
+        m = __hmax2(m, __hmax2(am(a.x, a.y), am(a.z, a.w)));
     }
     // |x| as a non-negative fp32 bit pattern orders like an unsigned integer
     float f = fmaxf(__low2float(m), __high2float(m));
@@ -73,9 +84,10 @@ __device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t
 }
 
 // grid: (blocks_per_head, n_heads).
+template <bool kHalf>
 __global__ void __launch_bounds__(kThreads)
 absmax_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, uint32_t* __restrict__ amax_bits) {
-    absmax_body(x, vecs_per_head, amax_bits);
+    absmax_body<kHalf>(x, vecs_per_head, amax_bits);
 }
 
 // two floats -> two e4m3 codes (lo in bits 0..7, hi in bits 8..15), RNE, saturating
@@ -85,17 +97,20 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
     return (uint32_t)r;
 }
 
+template <bool kHalf>
 __device__ __forceinline__ uint32_t quant4(uint32_t w0, uint32_t w1, float s) {
-    // w0, w1: four bf16 values; an fp32 with the bf16 bits in its upper half is that value
-    float a = __fdiv_rn(__uint_as_float(w0 << 16), s);
-    float b = __fdiv_rn(__uint_as_float(w0 & 0xffff0000u), s);
-    float c = __fdiv_rn(__uint_as_float(w1 << 16), s);
-    float e = __fdiv_rn(__uint_as_float(w1 & 0xffff0000u), s);
+    // w0, w1: four 16-bit values
+    using T = In16<kHalf>;
+    float a = __fdiv_rn(T::lo(w0), s);
+    float b = __fdiv_rn(T::hi(w0), s);
+    float c = __fdiv_rn(T::lo(w1), s);
+    float e = __fdiv_rn(T::hi(w1), s);
     return cvt_e4m3x2(a, b) | (cvt_e4m3x2(c, e) << 16);
 }
 
-// One block's share of head blockIdx.y.  Each thread turns 32 B of bf16 into 16 B
-// of e4m3 per step.  pairs_per_head = elems_per_head / 16.
+// One block's share of head blockIdx.y.  Each thread turns 32 B of 16-bit input into
+// 16 B of e4m3 per step.  pairs_per_head = elems_per_head / 16.
+template <bool kHalf>
 __device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64_t pairs_per_head,
                                               const float* __restrict__ scale_in,
                                               const uint32_t* __restrict__ amax_bits,
@@ -116,20 +131,21 @@ __device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64
         int64_t i = pairs_per_head - 1 - r;
         uint4 a = ld_nc_v4(xh + 2 * i), b = ld_nc_v4(xh + 2 * i + 1);
         uint4 o;
-        o.x = quant4(a.x, a.y, s);
-        o.y = quant4(a.z, a.w, s);
-        o.z = quant4(b.x, b.y, s);
-        o.w = quant4(b.z, b.w, s);
+        o.x = quant4<kHalf>(a.x, a.y, s);
+        o.y = quant4<kHalf>(a.z, a.w, s);
+        o.z = quant4<kHalf>(b.x, b.y, s);
+        o.w = quant4<kHalf>(b.z, b.w, s);
         oh[i] = o;
     }
 }
 
 // grid: (blocks_per_head, n_heads).
+template <bool kHalf>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const uint4* __restrict__ x, int64_t pairs_per_head,
                 const float* __restrict__ scale_in, const uint32_t* __restrict__ amax_bits,
                 uint4* __restrict__ out, float* __restrict__ scale_out) {
-    quantize_body(x, pairs_per_head, scale_in, amax_bits, out, scale_out);
+    quantize_body<kHalf>(x, pairs_per_head, scale_in, amax_bits, out, scale_out);
 }
 
 // All tensors of one attention call in two launches: blockIdx.z picks the tensor.
@@ -142,15 +158,17 @@ struct QuantBatch {
     float* scale_out[4];
 };
 
+template <bool kHalf>
 __global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch b) {
     const int z = blockIdx.z;
     if (b.amax_acc[z] != nullptr && b.pairs_per_head[z] > 0)
-        absmax_body(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
+        absmax_body<kHalf>(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
 }
 
+template <bool kHalf>
 __global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBatch b) {
     const int z = blockIdx.z;
-    quantize_body(b.x[z], b.pairs_per_head[z], nullptr, b.amax_in[z], b.out[z], b.scale_out[z]);
+    quantize_body<kHalf>(b.x[z], b.pairs_per_head[z], nullptr, b.amax_in[z], b.out[z], b.scale_out[z]);
 }
 
 }  // namespace
@@ -182,18 +200,22 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
     const unsigned bx = (unsigned)(want < have ? (want < 1 ? 1 : want) : (have < 1 ? 1 : have));
     if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
         return FP8ATTN_ERR_CUDA;
+    const bool half = (flags & FP8ATTN_INPUT_FP16) != 0;
     if (elems_train > 0) {
-        absmax_batch_kernel<<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
+        if (half) absmax_batch_kernel<true><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
+        else absmax_batch_kernel<false><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
         count_launch();
     }
-    quantize_batch_kernel<<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
+    if (half) quantize_batch_kernel<true><<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
+    else quantize_batch_kernel<false><<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
 }
 
 int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
                     const float* scale_in, void* x_fp8, float* scale_out,
-                    uint32_t* amax_bits, cudaStream_t stream) {
+                    uint32_t* amax_bits, uint32_t flags, cudaStream_t stream) {
+    const bool half = (flags & FP8ATTN_INPUT_FP16) != 0;
     if (n_heads <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     const int64_t vecs = elems_per_head / 8, pairs = elems_per_head / 16;
@@ -208,15 +230,21 @@ int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
         if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * n_heads, stream) != cudaSuccess)
             return FP8ATTN_ERR_CUDA;
         if (elems_per_head > 0) {
-            absmax_kernel<<<dim3(blocks_for((vecs + 3) / 4), (unsigned)n_heads), kThreads, 0, stream>>>(
-                (const uint4*)x_bf16, vecs, amax_bits);
+            const dim3 grid(blocks_for((vecs + 3) / 4), (unsigned)n_heads);
+            if (half) absmax_kernel<true><<<grid, kThreads, 0, stream>>>((const uint4*)x_bf16, vecs, amax_bits);
+            else absmax_kernel<false><<<grid, kThreads, 0, stream>>>((const uint4*)x_bf16, vecs, amax_bits);
             count_launch();
         }
     }
     // also launched for empty heads when the scale must be written out
     if (elems_per_head > 0 || scale_out != nullptr) {
-        quantize_kernel<<<dim3(blocks_for(pairs), (unsigned)n_heads), kThreads, 0, stream>>>(
-            (const uint4*)x_bf16, pairs, scale_in, amax_bits, (uint4*)x_fp8, scale_out);
+        const dim3 grid(blocks_for(pairs), (unsigned)n_heads);
+        if (half)
+            quantize_kernel<true><<<grid, kThreads, 0, stream>>>((const uint4*)x_bf16, pairs, scale_in,
+                                                                 amax_bits, (uint4*)x_fp8, scale_out);
+        else
+            quantize_kernel<false><<<grid, kThreads, 0, stream>>>((const uint4*)x_bf16, pairs, scale_in,
+                                                                  amax_bits, (uint4*)x_fp8, scale_out);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
@@ -284,6 +312,6 @@ extern "C" int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_
     int rc = static_amax_address(&amax);
     if (rc != FP8ATTN_OK) return rc;
     // launch_quantize clears the accumulators it uses at the start of every call
-    return launch_quantize(x_bf16, (int64_t)B * H, rows * (int64_t)d, scale_in, x_fp8, scale_out, amax,
+    return launch_quantize(x_bf16, (int64_t)B * H, rows * (int64_t)d, scale_in, x_fp8, scale_out, amax, 0u,
                            static_cast<cudaStream_t>(cuda_stream));
 }

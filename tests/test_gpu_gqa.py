@@ -67,6 +67,6 @@ def test_unknown_flag_is_rejected():
     o = torch.zeros((1, 1, 8, 64), dtype=torch.bfloat16, device="cuda")
     s = torch.ones((1, 1), dtype=torch.float32, device="cuda")
     p = lambda t: t.data_ptr()
-    rc = lib.fp8attn_icl_forward_ex(p(q), None, p(q), p(q), p(s), p(s), p(s), 1, 1, 8, 0, 64, 0.0, 2,
+    rc = lib.fp8attn_icl_forward_ex(p(q), None, p(q), p(q), p(s), p(s), p(s), 1, 1, 8, 0, 64, 0.0, 0x80,
                                     p(o), None, p(ws), ws.numel(), None)
     assert rc == api.ERR_INVALID_ARG
