@@ -763,12 +763,15 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     const int64_t grid = heads * (a.blocks_train + a.blocks_test);
     if (grid > 0x7fffffffll) return FP8ATTN_ERR_UNSUPPORTED;
     auto kern = icl_attention_kernel<kFp8, kD, kHalf>;
-    static bool attr_set = false;   // per instantiation
-    if (!attr_set) {
+    // the opt-in to large dynamic shared memory is per device (and per instantiation)
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return FP8ATTN_ERR_CUDA;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     kern<<<(unsigned)grid, kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test, mk, mv, a);
     count_launch();
