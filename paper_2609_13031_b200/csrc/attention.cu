@@ -1,7 +1,7 @@
 // Fused ICL attention for sm_100a: train->train and test->train in one launch.
 //
 // One CTA owns up to 256 query rows (two 128-row tiles) of one (b,h) and walks
-// over all train keys in steps of kKeys keys.  Warp roles (default build):
+// over all train keys in steps of kKeys keys.  Warp roles:
 //   warps 0-3   softmax of query tile 0, one row per thread
 //   warps 4-7   softmax of query tile 1
 //   warp  8     issues the Q K^T tcgen05.mma of both tiles (one elected lane)
@@ -14,8 +14,8 @@
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
-// probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 in the
-// 16-bit path) to its own tensor-memory region, from where it is the A operand
+// probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 / fp16 in
+// the 16-bit path) to its own tensor-memory region, from where it is the A operand
 // of O_t += P_t V.  Where 512 columns cannot hold a separate P (bf16, d = 128),
 // P is written over S and Q K^T waits for P V instead.  The FP8 d = 128 path
 // steps over 96 keys at a time to make room for P.
