@@ -223,3 +223,28 @@ def test_fp8_degenerate_heads_zero_queries_zero_keys_and_saturated_test_queries(
         A, Abs, Bnd = oracle.icl_attention_rows(q8, z["k8"], z["v8"], np.arange(nq), sq=z["sq"], sk=z["sk"],
                                                 sv=z["sv"])
         check_fp8_attention(out_to_f64(out), A, Abs, Bnd, diffuse=False, label=name, named_config=False)
+
+
+@pytest.mark.parametrize("d,fp8", [(128, True), (64, True), (128, False), (64, False)])
+def test_repeated_launches_are_bit_identical(d, fp8):
+    """Every barrier hand-over in the kernel orders real data: a race would show up as
+    run-to-run differences, so the same call must give the same bits every time."""
+    torch.manual_seed(d + fp8)
+    B, H, N, M = 1, 4, 12000, 3000
+    ws = api.new_workspace(B, H)
+    if fp8:
+        mk = lambda r: torch.randint(0, 256, (B, H, r, d), dtype=torch.uint8, device="cuda")
+        clean = lambda t: torch.where((t & 0x7F) == 0x7F, t & 0xFE, t)       # no NaN codes
+        q, t, k, v = (clean(mk(r)) for r in (N, M, N, N))
+        s = torch.full((B, H), 0.003, dtype=torch.float32, device="cuda")
+        run = lambda: api.icl_forward_fp8(q, t, k, v, s, s, s, ws)
+    else:
+        mk = lambda r: torch.randn((B, H, r, d), dtype=torch.bfloat16, device="cuda")
+        q, t, k, v = mk(N), mk(M), mk(N), mk(N)
+        run = lambda: api.icl_forward_bf16(q, t, k, v, ws)
+    first = [o.clone() for o in run()]
+    assert all(torch.isfinite(o.float()).all() for o in first)
+    for _ in range(6):
+        again = run()
+        assert torch.equal(again[0], first[0]) and torch.equal(again[1], first[1])
+    assert api.last_device_status(ws) == (0, 0)
