@@ -48,3 +48,49 @@ def test_dispatch_gate_matches_the_paper_constant():
     assert api.GATE_TRAIN_ROWS == gate
     assert not api.gate_use_fp8(gate) and api.gate_use_fp8(gate + 1)
     assert not api.gate_use_fp8(1) and api.gate_use_fp8(1 << 20)
+
+
+def test_argument_checks_run_on_the_host_before_anything_touches_a_gpu():
+    """Every entry point validates its arguments first, so the error codes can be checked on
+    a machine without a GPU.  Pointers here are fake, suitably aligned addresses: a call that
+    fails validation must not dereference or launch anything."""
+    import pytest
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("fake pointers are only ever passed where no GPU could be reached")
+    lib = api.load()
+    P, WS = 0x10000, 0x20000                      # 16- and 256-byte aligned fake device addresses
+    ws_bytes = api.workspace_bytes(1, 2)
+    q = lambda *a: lib.fp8attn_quantize(*a)
+    # shape and pointer checks of the quantizer
+    assert q(P, 0, 2, 8, 64, None, P, P, WS, ws_bytes, None) == api.ERR_INVALID_ARG      # B = 0
+    assert q(P, 1, 2, 8, 96, None, P, P, WS, ws_bytes, None) == api.ERR_UNSUPPORTED      # d = 96
+    assert q(P, 1, 2, -1, 64, None, P, P, WS, ws_bytes, None) == api.ERR_INVALID_ARG     # rows < 0
+    assert q(None, 1, 2, 8, 64, None, P, P, WS, ws_bytes, None) == api.ERR_INVALID_ARG   # no input
+    assert q(P + 2, 1, 2, 8, 64, None, P, P, WS, ws_bytes, None) == api.ERR_INVALID_ARG  # misaligned
+    assert q(P, 1, 2, 8, 64, None, P, None, WS, ws_bytes, None) == api.ERR_INVALID_ARG   # no scale at all
+    assert q(P, 1, 2, 8, 64, None, P, P, None, ws_bytes, None) == api.ERR_WORKSPACE
+    assert q(P, 1, 2, 8, 64, None, P, P, WS + 16, ws_bytes, None) == api.ERR_WORKSPACE   # misaligned
+    assert q(P, 1, 2, 8, 64, None, P, P, WS, ws_bytes - 1, None) == api.ERR_WORKSPACE    # too small
+    assert lib.fp8attn_quantize_ex(P, 1, 2, 8, 64, None, P, P, 0x40, WS, ws_bytes, None) == api.ERR_INVALID_ARG
+    # the fused forward
+    f = lambda *a: lib.fp8attn_icl_forward(*a)
+    ok = [P, P, P, P, P, P, P, 1, 2, 8, 4, 64, 0.0, P, P, WS, ws_bytes, None]
+    def bad(i, v):
+        a = list(ok)
+        a[i] = v
+        return f(*a)
+    assert bad(0, None) == api.ERR_INVALID_ARG         # train queries missing
+    assert bad(1, None) == api.ERR_INVALID_ARG         # test queries missing although n_test > 0
+    assert bad(4, None) == api.ERR_INVALID_ARG         # a scale missing
+    assert bad(9, 0) == api.ERR_INVALID_ARG            # n_train = 0
+    assert bad(10, -1) == api.ERR_INVALID_ARG          # n_test < 0
+    assert bad(11, 256) == api.ERR_UNSUPPORTED         # head dimension
+    assert bad(12, float("nan")) == api.ERR_INVALID_ARG
+    assert bad(14, None) == api.ERR_INVALID_ARG        # test output missing
+    assert bad(16, 0) == api.ERR_WORKSPACE
+    # allocation-free quantizer: its own size limit
+    assert lib.fp8attn_quantize_noalloc(P, 1, api.NOALLOC_MAX_HEADS + 1, 8, 64, None, P, P, None) == api.ERR_TOO_LARGE
+    # arguments in order, but no GPU: the call reports it; nothing falls back to the CPU
+    assert f(*ok) in (api.ERR_CUDA, api.ERR_UNSUPPORTED)
+    assert q(P, 1, 2, 8, 64, None, P, P, WS, ws_bytes, None) in (api.ERR_CUDA, api.ERR_UNSUPPORTED)
