@@ -99,8 +99,15 @@ int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, cons
  * the flag the scale comes from the train queries alone (the paper's proposal).
  * The "per-call query scale" ablation arm needs no flag: quantize the test
  * queries with fp8attn_quantize and scale_in = NULL.
- * FP8ATTN_INPUT_FP16 (above): all four inputs are IEEE fp16. */
+ * FP8ATTN_INPUT_FP16 (above): all four inputs are IEEE fp16.
+ * FP8ATTN_SCALES_GIVEN: scale_q, scale_k and scale_v are INPUTS, e.g. amax/448 with
+ * the per-head maxima taken in the epilogue of the projection that produced Q, K
+ * and V (the paper's method section notes that the quantization overhead is what
+ * limits small tables).  No maximum pass runs: one launch, each element read
+ * once; values outside a given scale's range saturate at +-448.  Not combinable
+ * with FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS. */
 #define FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS 1u
+#define FP8ATTN_SCALES_GIVEN 4u
 int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test,
                             int B, int H, int64_t n_train, int64_t n_test, int d,
                             void* q_train_fp8, void* k_fp8, void* v_fp8, void* q_test_fp8,

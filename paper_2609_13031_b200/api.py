@@ -29,6 +29,7 @@ EXPORTS = (
 # flags of fp8attn_quantize_ex / fp8attn_quantize_qkv_ex
 QUERY_SCALE_FROM_ALL_ROWS = 1
 INPUT_FP16 = 2
+SCALES_GIVEN = 4
 # flags of fp8attn_icl_forward_ex / bf16attn_icl_forward_ex
 TEST_ROWS_USE_KV_HEAD0 = 1
 TEST_ROWS_ONLY = 2
@@ -182,7 +183,10 @@ def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor
 def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
     """fp8attn_quantize_qkv: all four quantizations of one attention call in two
     launches.  Returns dict(q8, k8, v8, t8, sq, sk, sv); ``out`` may supply those
-    tensors preallocated."""
+    tensors preallocated.  With SCALES_GIVEN, ``out`` must hold sq, sk, sv and they
+    are read instead of written (one launch)."""
+    if flags & SCALES_GIVEN:
+        assert out is not None and all(n in out for n in ("sq", "sk", "sv"))
     B, H, n_train, d = _dims(k)
     n_test = 0 if q_test is None else q_test.shape[2]
     dev = k.device

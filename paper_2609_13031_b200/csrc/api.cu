@@ -109,7 +109,9 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS | FP8ATTN_INPUT_FP16))
+    if (flags & ~(uint32_t)(FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS | FP8ATTN_INPUT_FP16 | FP8ATTN_SCALES_GIVEN))
+        return FP8ATTN_ERR_INVALID_ARG;
+    if ((flags & FP8ATTN_SCALES_GIVEN) && (flags & FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS))
         return FP8ATTN_ERR_INVALID_ARG;
     if (!q_train || !k || !v || !q_train_fp8 || !k_fp8 || !v_fp8 || !scale_q || !scale_k || !scale_v)
         return FP8ATTN_ERR_INVALID_ARG;

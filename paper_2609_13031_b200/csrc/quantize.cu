@@ -153,6 +153,7 @@ struct QuantBatch {
     const uint4* x[4];
     uint4* out[4];
     int64_t pairs_per_head[4];
+    const float* scale_in[4];     // given scales (NULL: derive the scale from amax_in)
     const uint32_t* amax_in[4];   // accumulators the scale is derived from
     uint32_t* amax_acc[4];        // accumulators this tensor's maximum goes to (NULL: none)
     float* scale_out[4];
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch
 template <bool kHalf>
 __global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBatch b) {
     const int z = blockIdx.z;
-    quantize_body<kHalf>(b.x[z], b.pairs_per_head[z], nullptr, b.amax_in[z], b.out[z], b.scale_out[z]);
+    quantize_body<kHalf>(b.x[z], b.pairs_per_head[z], b.scale_in[z], b.amax_in[z], b.out[z], b.scale_out[z]);
 }
 
 }  // namespace
@@ -193,15 +194,23 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
         // single-call form: the query scale covers train and test queries alike
         if (z == 3 && (flags & FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS) && elems_test > 0) b.amax_acc[z] = amax_bits;
         b.scale_out[z] = scales[z];
+        b.scale_in[z] = nullptr;
+        if (flags & FP8ATTN_SCALES_GIVEN) {
+            // scales computed upstream: nothing to reduce, nothing to write back
+            b.scale_in[z] = scales[z == 3 ? 0 : z];
+            b.scale_out[z] = nullptr;
+            b.amax_acc[z] = nullptr;
+        }
     }
     const int tensors = elems_test > 0 ? 4 : 3;
     const int64_t want = (148 * 16 + n_heads * 3 - 1) / (n_heads * 3);
     const int64_t have = (elems_train / 16 + kThreads - 1) / kThreads;
     const unsigned bx = (unsigned)(want < have ? (want < 1 ? 1 : want) : (have < 1 ? 1 : have));
-    if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
+    if (!(flags & FP8ATTN_SCALES_GIVEN) &&
+        cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
         return FP8ATTN_ERR_CUDA;
     const bool half = (flags & FP8ATTN_INPUT_FP16) != 0;
-    if (elems_train > 0) {
+    if (elems_train > 0 && !(flags & FP8ATTN_SCALES_GIVEN)) {
         if (half) absmax_batch_kernel<true><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
         else absmax_batch_kernel<false><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
         count_launch();

@@ -179,3 +179,40 @@ def test_fp16_flags_are_checked():
     assert rc == api.ERR_INVALID_ARG
     rc = lib.fp8attn_quantize_ex(p(x), 1, 1, 8, 64, None, p(o), p(s), api.INPUT_FP16, p(ws), ws.numel(), None)
     assert rc == api.OK
+
+
+# ---- scales computed upstream ----------------------------------------------------------
+
+def test_quantize_with_given_scales_is_one_launch_and_bit_exact():
+    w = W.CONFIGS["C2"].scaled(1031, 77)
+    g = W.generate(w)
+    ref = quantized(g)
+    ws = api.new_workspace(w.B, w.H)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    x = {k: bf16_dev(g[k]) for k in ("q_train", "q_test", "k", "v")}
+    # the scales the maximum pass would have found: identical codes, in one launch
+    given = {"sq": dev(ref[4]), "sk": dev(ref[5]), "sv": dev(ref[6])}
+    before = api.launch_count()
+    o = api.quantize_qkv(x["q_train"], x["k"], x["v"], x["q_test"], ws, out=dict(given),
+                         flags=api.SCALES_GIVEN)
+    assert api.launch_count() - before == 1
+    for name, r in zip(("q8", "t8", "k8", "v8"), ref[:4]):
+        assert np.array_equal(o[name].cpu().numpy(), r), name
+    for name, r in zip(("sq", "sk", "sv"), ref[4:]):
+        assert np.array_equal(o[name].cpu().numpy(), r), name          # left as given
+    # other scales: the oracle with the same scales, values out of range saturate
+    half = {k: dev(v / 2) for k, v in zip(("sq", "sk", "sv"), ref[4:])}
+    o = api.quantize_qkv(x["q_train"], x["k"], x["v"], x["q_test"], ws, out=dict(half),
+                         flags=api.SCALES_GIVEN)
+    for name, src, sc in (("q8", "q_train", 4), ("t8", "q_test", 4), ("k8", "k", 5), ("v8", "v", 6)):
+        want, _ = oracle.quantize(g[src], scale_in=ref[sc] / 2)
+        assert np.array_equal(o[name].cpu().numpy(), want), name
+    assert (o["k8"].cpu().numpy() & 0x7F).max() == 0x7E
+    assert api.last_device_status(ws) == (0, 0)
+    lib = api.load()
+    p = lambda t: t.data_ptr()
+    rc = lib.fp8attn_quantize_qkv_ex(p(x["q_train"]), p(x["k"]), p(x["v"]), p(x["q_test"]), w.B, w.H,
+                                     w.n_train, w.n_test, w.d, p(o["q8"]), p(o["k8"]), p(o["v8"]), p(o["t8"]),
+                                     p(o["sq"]), p(o["sk"]), p(o["sv"]),
+                                     api.SCALES_GIVEN | api.QUERY_SCALE_FROM_ALL_ROWS, p(ws), ws.numel(), None)
+    assert rc == api.ERR_INVALID_ARG
