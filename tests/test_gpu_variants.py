@@ -216,3 +216,31 @@ def test_quantize_with_given_scales_is_one_launch_and_bit_exact():
                                      p(o["sq"]), p(o["sk"]), p(o["sv"]),
                                      api.SCALES_GIVEN | api.QUERY_SCALE_FROM_ALL_ROWS, p(ws), ws.numel(), None)
     assert rc == api.ERR_INVALID_ARG
+
+
+def test_fp16_whole_path_at_size_sampled():
+    """fp16 in, fp16 out at a size that spans many CTAs, steps and a ragged tail: the
+    quantizer bit-exact, the FP8 attention and the fp16 twin against the oracle on
+    sampled rows."""
+    from helpers import sample_rows
+    w = W.CONFIGS["C3"].scaled(20011, 3001)
+    g = {k: to_fp16_bits(v) for k, v in W.generate(w).items()}
+    x = {k: fp16_dev(v) for k, v in g.items()}
+    ws = api.new_workspace(w.B, w.H)
+    q8, t8, k8, v8, sq, sk, sv = quantized(g, "fp16")
+    o = api.quantize_qkv(x["q_train"], x["k"], x["v"], x["q_test"], ws)
+    for name, r in zip(("q8", "t8", "k8", "v8", "sq", "sk", "sv"), (q8, t8, k8, v8, sq, sk, sv)):
+        assert np.array_equal(o[name].cpu().numpy(), r), name
+    f_tr, f_te = api.icl_attention(x["q_train"], x["q_test"], x["k"], x["v"], ws)
+    h_tr, h_te = api.icl_forward_bf16(x["q_train"], x["q_test"], x["k"], x["v"], ws)
+    assert f_tr.dtype == torch.float16 and h_te.dtype == torch.float16
+    assert api.last_device_status(ws) == (0, 0)
+    for name, f_out, h_out, codes, bits, nq in (("train", f_tr, h_tr, q8, g["q_train"], w.n_train),
+                                                ("test", f_te, h_te, t8, g["q_test"], w.n_test)):
+        rows = sample_rows(nq, 40, 9)
+        idx = torch.from_numpy(rows).cuda()
+        A, Abs, Bnd = oracle.icl_attention_rows(codes, k8, v8, rows, sq=sq, sk=sk, sv=sv)
+        check_fp8_attention(f64(f_out[:, :, idx]), A, Abs, Bnd, diffuse=False, label=f"fp16-io/{name}",
+                            named_config=False)
+        A, Abs, _ = oracle.icl_attention_rows(bits, g["k"], g["v"], rows, dtype16="fp16")
+        check_bf16_attention(f64(h_out[:, :, idx]), A, Abs, label=f"fp16-twin/{name}", rounding=2.0 ** -12)
