@@ -236,7 +236,10 @@ def main():
     dev = {k: torch.empty_like(v, device="cuda") for k, v in host.items()}
     for k in host:
         dev[k].copy_(host[k], non_blocking=True)
-    ws = api.new_workspace(w.B, w.H)
+    # sized for FP8ATTN_SPLIT_TAIL, which both attention paths run with (it acts only on launches of
+    # fewer than 8 CTAs per SM: C1 and C2 here; C3-C5 run exactly as without it)
+    ws = api.new_workspace(w.B, w.H, n_train=w.n_train, n_test=w.n_test, d=w.d)
+    fwd_flags = api.SPLIT_TAIL
     shape_tr, shape_te = (w.B, w.H, w.n_train, w.d), (w.B, w.H, w.n_test, w.d)
     buf = {
         "q8": torch.empty(shape_tr, dtype=torch.uint8, device="cuda"),
@@ -259,11 +262,11 @@ def main():
 
     def attention_fp8():
         api.icl_forward_fp8(buf["q8"], buf["t8"], buf["k8"], buf["v8"], buf["sq"], buf["sk"], buf["sv"],
-                            ws, 0.0, out_train=buf["o_tr"], out_test=buf["o_te"])
+                            ws, 0.0, out_train=buf["o_tr"], out_test=buf["o_te"], flags=fwd_flags)
 
     def attention_bf16():
         api.icl_forward_bf16(dev["q_train"], dev["q_test"], dev["k"], dev["v"], ws, 0.0,
-                             out_train=buf["o_tr"], out_test=buf["o_te"])
+                             out_train=buf["o_tr"], out_test=buf["o_te"], flags=fwd_flags)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -369,7 +372,7 @@ def main():
                 api.quantize_qkv(d_in["q_train"], d_in["k"], d_in["v"], d_in["q_test"], ws, out=d_buf)
                 api.icl_forward_fp8(d_buf["q8"], d_buf["t8"], d_buf["k8"], d_buf["v8"], d_buf["sq"],
                                     d_buf["sk"], d_buf["sv"], ws, 0.0, out_train=d_buf["o_tr"],
-                                    out_test=d_buf["o_te"])
+                                    out_test=d_buf["o_te"], flags=fwd_flags)
                 e_c = torch.cuda.Event()
                 e_c.record(s_cmp)
                 free_in[i % 2] = e_c
@@ -431,7 +434,7 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
             "data": "synthetic",
             "config": {"workload": workload_label(w),
-                       "step": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward",
+                       "step": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
                        "l2": "inputs larger than L2 (bf16 inputs %.0f MB)" % (h2d / 1e6),
                        "replicas": world},
             "clocks": clocks,

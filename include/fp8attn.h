@@ -175,11 +175,28 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
  * fp8attn_icl_forward_ex, and the inputs, the on-chip probabilities and the
  * outputs of bf16attn_icl_forward_ex (which then is an fp16 kernel).
  *
+ * FP8ATTN_SPLIT_TAIL balances the last, partly filled round of the launch.  The
+ * grid is one CTA per 256 query rows of a head; when the number of CTAs is not
+ * a multiple of the number of SMs, the CTAs left over after the last full
+ * round would run alone on a fraction of the GPU.  With this flag each of them
+ * is replaced by up to 16 CTAs that share its query rows and divide the train
+ * keys between them, followed by a small kernel that combines their partial
+ * results (the online softmax of the paper's kernel, applied once more across
+ * key ranges).  The workspace must then be at least
+ * fp8attn_workspace_bytes(B, H, n_train, n_test, d) with n_train > 0, which
+ * includes the scratch for the partial results, else
+ * FP8ATTN_ERR_WORKSPACE.  The split is applied only where it was measured to
+ * pay (launches of fewer than 8 CTAs per SM whose key ranges keep at least
+ * four steps); elsewhere the flag changes nothing.  Results stay within the same tolerances, but which
+ * rows take the split path depends on the sizes of the call, so a row's result
+ * is no longer bit-identical across calls with different n_test.
+ *
  * Unknown flag bits return FP8ATTN_ERR_INVALID_ARG.  flags = 0 is the plain call.
  */
 #define FP8ATTN_TEST_ROWS_USE_KV_HEAD0 1u
 #define FP8ATTN_TEST_ROWS_ONLY 2u
 #define FP8ATTN_IO_FP16 4u
+#define FP8ATTN_SPLIT_TAIL 8u
 int fp8attn_icl_forward_ex(const void* q_train_fp8, const void* q_test_fp8,
                            const void* k_fp8, const void* v_fp8,
                            const float* scale_q, const float* scale_k, const float* scale_v,
@@ -254,7 +271,11 @@ int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int
                              const float* scale_in, void* x_fp8, float* scale_out,
                              void* cuda_stream);
 
-/* Bytes of workspace the three calls above need for these sizes (a few KB). */
+/* Bytes of workspace the calls above need: a few KB for the status words and the
+ * per-head accumulators (all that is returned for n_train = 0), plus, for
+ * n_train > 0 and d in {64, 128}, the scratch of FP8ATTN_SPLIT_TAIL (about 13 MB
+ * at d = 64, 26 MB at d = 128; independent of n_train and n_test).  A workspace
+ * of the smaller size serves every call that does not set that flag. */
 size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t n_test, int d);
 
 /* Synchronises `cuda_stream`, reads and clears the device status word of

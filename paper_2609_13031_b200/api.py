@@ -34,6 +34,7 @@ SCALES_GIVEN = 4
 TEST_ROWS_USE_KV_HEAD0 = 1
 TEST_ROWS_ONLY = 2
 IO_FP16 = 4
+SPLIT_TAIL = 8
 GATE_TRAIN_ROWS = 8192
 
 _lib = None
@@ -126,9 +127,11 @@ def workspace_bytes(B: int, H: int, n_train: int = 0, n_test: int = 0, d: int = 
     return int(load().fp8attn_workspace_bytes(B, H, n_train, n_test, d))
 
 
-def new_workspace(B: int, H: int, device="cuda") -> torch.Tensor:
-    """A zero-filled workspace tensor for tensors with B*H heads."""
-    return torch.zeros(workspace_bytes(B, H), dtype=torch.uint8, device=device)
+def new_workspace(B: int, H: int, device="cuda", n_train: int = 0, n_test: int = 0,
+                  d: int = 64) -> torch.Tensor:
+    """A zero-filled workspace tensor for tensors with B*H heads.  Given the sizes of an
+    attention call (n_train > 0) it also holds the scratch that SPLIT_TAIL needs."""
+    return torch.zeros(workspace_bytes(B, H, n_train, n_test, d), dtype=torch.uint8, device=device)
 
 
 def _dims(x: torch.Tensor):
@@ -323,17 +326,19 @@ def last_device_status(workspace: torch.Tensor):
     return int(rc), int(detail.value)
 
 
-def icl_attention(q_train, q_test, k, v, workspace=None, softmax_scale: float = 0.0):
+def icl_attention(q_train, q_test, k, v, workspace=None, softmax_scale: float = 0.0, flags: int = 0):
     """The whole hot path on bf16 inputs: quantize Q_train, K, V per head, quantize
-    Q_test with the train-query scale, then the fused FP8 attention."""
-    B, H, _, _ = _dims(k)
+    Q_test with the train-query scale, then the fused FP8 attention (``flags``: forward
+    flags, e.g. SPLIT_TAIL)."""
+    B, H, n_train, d = _dims(k)
     if workspace is None:
-        workspace = new_workspace(B, H, k.device)
+        workspace = new_workspace(B, H, k.device, n_train=n_train if flags & SPLIT_TAIL else 0, d=d)
     has_test = q_test is not None and q_test.shape[2] > 0
     o = quantize_qkv(q_train, k, v, q_test if has_test else None, workspace)
     q8, k8, v8, sq, sk, sv = o["q8"], o["k8"], o["v8"], o["sq"], o["sk"], o["sv"]
     t8 = o["t8"] if has_test else None
-    return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale, out_dtype=k.dtype)
+    return icl_forward_fp8(q8, t8, k8, v8, sq, sk, sv, workspace, softmax_scale, flags=flags,
+                           out_dtype=k.dtype)
 
 
 def icl_attention_arms(q_train, q_test, k, v, fp8_train: bool, fp8_test: bool, workspace=None,

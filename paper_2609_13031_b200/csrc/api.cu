@@ -41,7 +41,8 @@ int forward(bool fp8, const void* q_train, const void* q_test, const void* k, co
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0 || n_train > 0x7fffff00ll || n_test > 0x7fffff00ll)
         return FP8ATTN_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(FP8ATTN_TEST_ROWS_USE_KV_HEAD0 | FP8ATTN_TEST_ROWS_ONLY | FP8ATTN_IO_FP16))
+    if (flags & ~(uint32_t)(FP8ATTN_TEST_ROWS_USE_KV_HEAD0 | FP8ATTN_TEST_ROWS_ONLY | FP8ATTN_IO_FP16 |
+                            FP8ATTN_SPLIT_TAIL))
         return FP8ATTN_ERR_INVALID_ARG;
     const bool test_only = (flags & FP8ATTN_TEST_ROWS_ONLY) != 0;
     if (test_only && n_test < 1) return FP8ATTN_ERR_INVALID_ARG;
@@ -55,9 +56,17 @@ int forward(bool fp8, const void* q_train, const void* q_test, const void* k, co
     if (!(softmax_scale == softmax_scale) || isinf(softmax_scale)) return FP8ATTN_ERR_INVALID_ARG;
     rc = check_workspace(workspace, workspace_bytes_, B, H);
     if (rc != FP8ATTN_OK) return rc;
+    if ((flags & FP8ATTN_SPLIT_TAIL) && workspace_bytes_ < workspace_bytes(B, H) + split_scratch_bytes(d))
+        return FP8ATTN_ERR_WORKSPACE;
     rc = check_device();
     if (rc != FP8ATTN_OK) return rc;
     AttnParams p;
+    p.partial = nullptr;
+    p.partial_bytes = 0;
+    if (flags & FP8ATTN_SPLIT_TAIL) {
+        p.partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + workspace_bytes(B, H));
+        p.partial_bytes = workspace_bytes_ - workspace_bytes(B, H);
+    }
     p.q_train = q_train; p.q_test = q_test; p.k = k; p.v = v;
     p.scale_q = sq; p.scale_k = sk; p.scale_v = sv;
     p.B = B; p.H = H; p.n_train = n_train; p.n_test = n_test; p.d = d;
@@ -206,8 +215,10 @@ int fp8attn_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, uint
 
 int fp8attn_gate_use_fp8(int64_t n_train) { return n_train > FP8ATTN_GATE_TRAIN_ROWS ? 1 : 0; }
 
-size_t fp8attn_workspace_bytes(int B, int H, int64_t, int64_t, int) {
+size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t, int d) {
     if (B <= 0 || H <= 0) return 0;
+    // with the size of an attention call: room for the tail split's partial results as well
+    if (n_train > 0 && (d == 64 || d == 128)) return workspace_bytes(B, H) + split_scratch_bytes(d);
     return workspace_bytes(B, H);
 }
 

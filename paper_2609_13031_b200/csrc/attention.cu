@@ -46,6 +46,7 @@ constexpr int kRegsOther = 56;
 static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kNumThreads * kLaunchRegs,
               "setmaxnreg budgets exceed the CTA's register pool");
 constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxSplits = 16;        // key ranges a split query block is divided into, at most
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 // detail codes written next to FP8ATTN_ERR_TIMEOUT
@@ -308,6 +309,9 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) 
 constexpr uint32_t kSFreeBarrier0 = 1, kPFullBarrier0 = 3;
 constexpr uint32_t kSignalThreads = 128 + 32;   // one tile's softmax threads + the issuer warp
 
+// floats per row of a partial result: kD values of O, c*m, l, and padding to 16 bytes
+template <int kD> constexpr int kPartialStride = kD + 4;
+
 struct KernelArgs {
     const float* scale_q; const float* scale_k; const float* scale_v;
     void* out_train; void* out_test;
@@ -316,11 +320,18 @@ struct KernelArgs {
     int heads;                       // H, to find head 0 of a table
     int test_kv_head0;               // test rows read K, V and their scales from head 0 of their table
     int out_half;                    // FP8 kernel: outputs are IEEE fp16 instead of bf16
+    // Tail split: the query blocks from full_blocks on (the part of the grid that would
+    // fill less than one CTA per SM) are each run by `splits` CTAs over disjoint key ranges;
+    // those CTAs write unnormalised partial results to `partial`, combined afterwards.
+    int full_blocks, splits;
+    float* partial;                  // [unit][split][256 rows][kD + 4] fp32: O, c*m, l, pad
     float softmax_scale;
     uint32_t* status;
 };
 
-template <bool kFp8, int kD, bool kHalf>
+// kSplit: this launch runs the split query blocks (see KernelArgs); kept out of the main
+// instantiation, whose softmax warps have no register to spare for the extra indices.
+template <bool kFp8, int kD, bool kHalf, bool kSplit>
 __global__ void __launch_bounds__(kNumThreads, 1)
 icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                      const __grid_constant__ CUtensorMap map_q_test,
@@ -340,14 +351,20 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
 
     // ---- which query block is this CTA's ----
     const int blocks_per_head = args.blocks_train + args.blocks_test;
-    const int bh = blockIdx.x / blocks_per_head;
-    const int blk = blockIdx.x % blocks_per_head;
+    const int vblk = kSplit ? args.full_blocks + (int)blockIdx.x / args.splits : (int)blockIdx.x;
+    const int split = kSplit ? (int)blockIdx.x % args.splits : 0;
+    const int nsplit = kSplit ? args.splits : 1;
+    const int bh = vblk / blocks_per_head;
+    const int blk = vblk % blocks_per_head;
     const bool is_test = blk >= args.blocks_train;
     const int64_t q_rows = is_test ? args.n_test : args.n_train;
     const int64_t row0 = (int64_t)(is_test ? blk - args.blocks_train : blk) * (2 * kTileM);
     const int ntiles = (q_rows - row0 > kTileM) ? 2 : 1;
     const int64_t n_keys = args.n_train;
-    const int nkv = (int)((n_keys + kKeys - 1) / kKeys);
+    // this CTA's key steps: [j0, j0 + nkv) of the nkv_all steps over the train keys
+    const int nkv_all = (int)((n_keys + kKeys - 1) / kKeys);
+    const int j0 = (int)((int64_t)split * nkv_all / nsplit);
+    const int nkv = (int)((int64_t)(split + 1) * nkv_all / nsplit) - j0;
     const CUtensorMap* map_q = is_test ? &map_q_test : &map_q_train;
     // grouped-query variant: every test query head attends to the first K/V head of its table
     const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
@@ -408,14 +425,14 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 mbar_arrive_expect_tx(smem_u32(&bars.k_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
                     tma_load_3d(sK + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_k,
-                                b * C::kBoxCols, j * kKeys, bh_kv, smem_u32(&bars.k_full[s]));
+                                b * C::kBoxCols, (j0 + j) * kKeys, bh_kv, smem_u32(&bars.k_full[s]));
             }
             w.wait<400>(smem_u32(&bars.v_empty[s]), ph ^ 1, kWaitVEmpty);
             if (elect_one()) {
                 mbar_arrive_expect_tx(smem_u32(&bars.v_full[s]), C::kKVTileBytes);
                 for (int b = 0; b < C::kBoxes; ++b)
                     tma_load_3d(sV + s * C::kKVTileBytes + b * kKeys * C::kBoxBytes, &map_v,
-                                b * C::kBoxCols, j * kKeys, bh_kv, smem_u32(&bars.v_full[s]));
+                                b * C::kBoxCols, (j0 + j) * kKeys, bh_kv, smem_u32(&bars.v_full[s]));
             }
             __syncwarp();
         }
@@ -542,7 +559,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
                 }
                 FP8ATTN_STAMP(t * 8 + 1, j);
-                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)j * kKeys);
+                const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)(j0 + j) * kKeys);
                 if (valid < kKeys) {
 #pragma unroll
                     for (int i = 0; i < kKeys; ++i)
@@ -693,6 +710,25 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             w.wait(smem_u32(&bars.o_full[t]), 0, kWaitOFull);
             tc_fence_after_sync();
             const int64_t row = row0 + t * kTileM + row_in_tile;
+            if (kSplit) {
+                // partial result of this key range: unnormalised O, the reference maximum in
+                // exp2 units and the row sum; the combine kernel weighs and normalises
+                float* dst = args.partial +
+                             ((size_t)((vblk - args.full_blocks) * nsplit + split) * (2 * kTileM) +
+                              (size_t)(t * kTileM + row_in_tile)) * kPartialStride<kD>;
+#pragma unroll
+                for (int q = 0; q < kD / 32; ++q) {
+                    uint32_t o[32];
+                    tmem_ld_x32(tO + q * 32, o);
+                    tmem_wait_ld_x32(o);
+                    if (!w.dead) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<uint4*>(dst + q * 32 + i) = make_uint4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                    }
+                }
+                if (!w.dead) *reinterpret_cast<float2*>(dst + kD) = make_float2(m * c, l);
+            } else {
             const float inv = sv_scale / l;
             const bool out_half = kFp8 ? args.out_half != 0 : kHalf;   // 16-bit type of the outputs
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
@@ -722,12 +758,64 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     }
                 }
             }
+            }
         }
     }
     // ---- teardown ----
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// Combines the partial results of the split query blocks: with M = max_s c*m_s,
+// out = s_v * sum_s 2^(c*m_s - M) O_s / sum_s 2^(c*m_s - M) l_s.  One thread per row and
+// eight output columns.
+template <int kD>
+__global__ void __launch_bounds__(256)
+combine_split_kernel(const KernelArgs args, int units, int out_half, int fp8) {
+    const int per_row = kD / 8;
+    const int64_t tid = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t unit = tid / (2 * kTileM * per_row);
+    if (unit >= units) return;
+    const int r = (int)(tid / per_row) % (2 * kTileM);
+    const int g = (int)(tid % per_row);
+    const int blocks_per_head = args.blocks_train + args.blocks_test;
+    const int vblk = args.full_blocks + (int)unit;
+    const int bh = vblk / blocks_per_head, blk = vblk % blocks_per_head;
+    const bool is_test = blk >= args.blocks_train;
+    const int64_t q_rows = is_test ? args.n_test : args.n_train;
+    const int64_t row = (int64_t)(is_test ? blk - args.blocks_train : blk) * (2 * kTileM) + r;
+    if (row >= q_rows) return;
+    const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
+    const float* base = args.partial + ((size_t)unit * args.splits * (2 * kTileM) + r) * kPartialStride<kD>;
+    const size_t split_stride = (size_t)(2 * kTileM) * kPartialStride<kD>;
+    float mmax = -INFINITY;
+    for (int s = 0; s < args.splits; ++s) mmax = fmaxf(mmax, base[s * split_stride + kD]);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float lsum = 0.f;
+    for (int s = 0; s < args.splits; ++s) {
+        const float* ps = base + s * split_stride;
+        const float wgt = exp2f(ps[kD] - mmax);
+        lsum = fmaf(wgt, ps[kD + 1], lsum);
+        const float4 a = *reinterpret_cast<const float4*>(ps + g * 8);
+        const float4 b = *reinterpret_cast<const float4*>(ps + g * 8 + 4);
+        acc[0] = fmaf(wgt, a.x, acc[0]); acc[1] = fmaf(wgt, a.y, acc[1]);
+        acc[2] = fmaf(wgt, a.z, acc[2]); acc[3] = fmaf(wgt, a.w, acc[3]);
+        acc[4] = fmaf(wgt, b.x, acc[4]); acc[5] = fmaf(wgt, b.y, acc[5]);
+        acc[6] = fmaf(wgt, b.z, acc[6]); acc[7] = fmaf(wgt, b.w, acc[7]);
+    }
+    const float inv = (fp8 ? args.scale_v[bh_kv] : 1.0f) / lsum;
+    uint4 v;
+    if (out_half) {
+        v.x = pack_f16x2(acc[0] * inv, acc[1] * inv); v.y = pack_f16x2(acc[2] * inv, acc[3] * inv);
+        v.z = pack_f16x2(acc[4] * inv, acc[5] * inv); v.w = pack_f16x2(acc[6] * inv, acc[7] * inv);
+    } else {
+        v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv); v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+        v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv); v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+    }
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
+                         ((int64_t)bh * q_rows + row) * kD;
+    *reinterpret_cast<uint4*>(out + g * 8) = v;
 }
 
 template <bool kFp8, int kD, bool kHalf>
@@ -760,21 +848,64 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     a.test_kv_head0 = (p.flags & FP8ATTN_TEST_ROWS_USE_KV_HEAD0) ? 1 : 0;
     a.out_half = (p.flags & FP8ATTN_IO_FP16) ? 1 : 0;
     a.status = p.status;
-    const int64_t grid = heads * (a.blocks_train + a.blocks_test);
+    int64_t grid = heads * (a.blocks_train + a.blocks_test);
     if (grid > 0x7fffffffll) return FP8ATTN_ERR_UNSUPPORTED;
-    auto kern = icl_attention_kernel<kFp8, kD, kHalf>;
-    // the opt-in to large dynamic shared memory is per device (and per instantiation)
-    static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    // Tail split: what is left of the grid after the last full round of one CTA per SM runs
+    // as several CTAs per query block, each over its own share of the keys.
+    a.full_blocks = (int)grid;
+    a.splits = 1;
+    a.partial = nullptr;
+    int units = 0;
+    if ((p.flags & FP8ATTN_SPLIT_TAIL) && p.partial != nullptr) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return FP8ATTN_ERR_CUDA;
+        const int64_t full = (grid / sms) * sms, left = grid - full;
+        const int64_t steps = (p.n_train + C::kKeys - 1) / C::kKeys;
+        // Measured: it pays from about one round up to about eight (1.37x at 1.1 rounds, 1.25x
+        // at 2.2, 1.1x at 4.3, nothing beyond 8), provided a key range keeps at least four
+        // steps; below that the two extra launches cost more than the split saves.
+        if (left > 0 && grid < 8 * (int64_t)sms && steps >= 16) {
+            int64_t splits = sms / left;
+            if (splits > steps / 4) splits = steps / 4;
+            if (splits > kMaxSplits) splits = kMaxSplits;
+            const size_t per_split = (size_t)left * 2 * kTileM * kPartialStride<kD> * sizeof(float);
+            while (splits >= 2 && per_split * (size_t)splits > p.partial_bytes) --splits;
+            if (splits >= 2) {
+                a.full_blocks = (int)full;
+                a.splits = (int)splits;
+                a.partial = p.partial;
+                units = (int)left;
+            }
+        }
+    }
+    auto kern = icl_attention_kernel<kFp8, kD, kHalf, false>;
+    auto kern_split = icl_attention_kernel<kFp8, kD, kHalf, true>;
+    // the opt-in to large dynamic shared memory is per device (and per instantiation)
+    static bool attr_set[64] = {};
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)C::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(kern_split, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)C::kSmemBytes) != cudaSuccess)
             return FP8ATTN_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<(unsigned)grid, kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test, mk, mv, a);
-    count_launch();
+    if (a.full_blocks > 0) {
+        kern<<<(unsigned)a.full_blocks, kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test, mk, mv, a);
+        count_launch();
+    }
+    if (units > 0) {
+        kern_split<<<(unsigned)(units * a.splits), kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test,
+                                                                                      mk, mv, a);
+        count_launch();
+        const int64_t threads = (int64_t)units * 2 * kTileM * (kD / 8);
+        combine_split_kernel<kD><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
+            a, units, kFp8 ? a.out_half : (kHalf ? 1 : 0), kFp8 ? 1 : 0);
+        count_launch();
+    }
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
 }
 

@@ -24,6 +24,10 @@ inline size_t workspace_bytes(int B, int H) {
     return kWsAmaxOffset + ((amax + 255) / 256) * 256;
 }
 
+// Scratch of the tail split (FP8ATTN_SPLIT_TAIL), appended to the workspace: partial results
+// of fewer than one CTA per SM, 256 rows of d + 4 floats each; sized for up to 192 SMs.
+inline size_t split_scratch_bytes(int d) { return (size_t)192 * 256 * (size_t)(d + 4) * sizeof(float); }
+
 void count_launch();
 
 // quantize.cu
@@ -50,6 +54,8 @@ struct AttnParams {
     uint32_t flags;    // FP8ATTN_* forward flags
     void* out_train; void* out_test;
     uint32_t* status;  // workspace status words
+    float* partial;    // scratch of the tail split (NULL: none)
+    size_t partial_bytes;
 };
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream);
 int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
