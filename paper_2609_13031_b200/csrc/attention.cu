@@ -369,6 +369,9 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     // grouped-query variant: every test query head attends to the first K/V head of its table
     const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
 
+    // the main launch does not depend on this one: let it start as soon as SMs are free
+    if (kSplit) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // A device error recorded earlier (and not yet read back by the host) is sticky:
     // nothing runs until fp8attn_last_device_status() has cleared it.
     if (*reinterpret_cast<volatile uint32_t*>(args.status) != 0u) return;
@@ -864,9 +867,10 @@ int launch(const AttnParams& p, cudaStream_t stream) {
             return FP8ATTN_ERR_CUDA;
         const int64_t full = (grid / sms) * sms, left = grid - full;
         const int64_t steps = (p.n_train + C::kKeys - 1) / C::kKeys;
-        // Measured: it pays from about one round up to about eight (1.37x at 1.1 rounds, 1.25x
-        // at 2.2, 1.1x at 4.3, nothing beyond 8), provided a key range keeps at least four
-        // steps; below that the two extra launches cost more than the split saves.
+        // Measured: it pays from about one round up to about eight (1.4x at 1.1 rounds, 1.27x
+        // at 2.2, 1.1x at 4.3, nothing beyond 8: after many rounds the SMs have drifted apart
+        // and the last round is no longer a round), provided a key range keeps at least four
+        // steps; below that the extra launches cost more than the split saves.
         if (left > 0 && grid < 8 * (int64_t)sms && steps >= 16) {
             int64_t splits = sms / left;
             if (splits > steps / 4) splits = steps / 4;
@@ -893,14 +897,30 @@ int launch(const AttnParams& p, cudaStream_t stream) {
             return FP8ATTN_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    if (a.full_blocks > 0) {
-        kern<<<(unsigned)a.full_blocks, kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test, mk, mv, a);
-        count_launch();
-    }
     if (units > 0) {
+        // The split blocks go first and release their dependents at once, and the main launch
+        // is allowed to start while they run (programmatic dependent launch): the two grids
+        // are independent, so the SMs the short split CTAs leave go straight to main CTAs.
         kern_split<<<(unsigned)(units * a.splits), kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test,
                                                                                       mk, mv, a);
         count_launch();
+    }
+    if (a.full_blocks > 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)a.full_blocks);
+        cfg.blockDim = dim3(kNumThreads);
+        cfg.dynamicSmemBytes = C::kSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = units > 0 ? 1 : 0;
+        if (cudaLaunchKernelEx(&cfg, kern, mq_train, mq_test, mk, mv, a) != cudaSuccess)
+            return FP8ATTN_ERR_CUDA;
+        count_launch();
+    }
+    if (units > 0) {
         const int64_t threads = (int64_t)units * 2 * kTileM * (kD / 8);
         combine_split_kernel<kD><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
             a, units, kFp8 ? a.out_half : (kHalf ? 1 : 0), kFp8 ? 1 : 0);
