@@ -56,7 +56,9 @@ enum : uint32_t {
 };
 
 // kFp8: e4m3 operands and P (else 16-bit operands and P).  kHalf: the 16-bit type of the
-// 16-bit kernel is IEEE fp16 instead of bf16 (ignored when kFp8).
+// call is IEEE fp16 instead of bf16: the outputs of both kernels, and the operands and P
+// of the 16-bit kernel.  (A run-time switch for the FP8 kernel's output type cost 4 % at
+// d = 64 through register allocation, hence a template parameter.)
 template <bool kFp8, int kD, bool kHalf = false>
 struct Cfg {
     static constexpr int kES = kFp8 ? 1 : 2;                    // element bytes
@@ -319,7 +321,6 @@ struct KernelArgs {
     int blocks_train, blocks_test;   // 256-row query blocks per head
     int heads;                       // H, to find head 0 of a table
     int test_kv_head0;               // test rows read K, V and their scales from head 0 of their table
-    int out_half;                    // FP8 kernel: outputs are IEEE fp16 instead of bf16
     // Tail split: the query blocks from full_blocks on (the part of the grid that would
     // fill less than one CTA per SM) are each run by `splits` CTAs over disjoint key ranges;
     // those CTAs write unnormalised partial results to `partial`, combined afterwards.
@@ -733,7 +734,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 if (!w.dead) *reinterpret_cast<float2*>(dst + kD) = make_float2(m * c, l);
             } else {
             const float inv = sv_scale / l;
-            const bool out_half = kFp8 ? args.out_half != 0 : kHalf;   // 16-bit type of the outputs
+            constexpr bool out_half = kHalf;   // 16-bit type of the outputs
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(is_test ? args.out_test : args.out_train) +
                                  ((int64_t)bh * q_rows + row) * kD;
 #pragma unroll
@@ -849,7 +850,6 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     a.softmax_scale = p.softmax_scale;
     a.heads = p.H;
     a.test_kv_head0 = (p.flags & FP8ATTN_TEST_ROWS_USE_KV_HEAD0) ? 1 : 0;
-    a.out_half = (p.flags & FP8ATTN_IO_FP16) ? 1 : 0;
     a.status = p.status;
     int64_t grid = heads * (a.blocks_train + a.blocks_test);
     if (grid > 0x7fffffffll) return FP8ATTN_ERR_UNSUPPORTED;
@@ -923,7 +923,7 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     if (units > 0) {
         const int64_t threads = (int64_t)units * 2 * kTileM * (kD / 8);
         combine_split_kernel<kD><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
-            a, units, kFp8 ? a.out_half : (kHalf ? 1 : 0), kFp8 ? 1 : 0);
+            a, units, kHalf ? 1 : 0, kFp8 ? 1 : 0);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
@@ -961,9 +961,12 @@ int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream
 }
 
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {
-    if (fp8) return p.d == 64 ? launch<true, 64, false>(p, stream) : launch<true, 128, false>(p, stream);
-    if (p.flags & FP8ATTN_IO_FP16)
-        return p.d == 64 ? launch<false, 64, true>(p, stream) : launch<false, 128, true>(p, stream);
+    const bool half = (p.flags & FP8ATTN_IO_FP16) != 0;
+    if (fp8) {
+        if (half) return p.d == 64 ? launch<true, 64, true>(p, stream) : launch<true, 128, true>(p, stream);
+        return p.d == 64 ? launch<true, 64, false>(p, stream) : launch<true, 128, false>(p, stream);
+    }
+    if (half) return p.d == 64 ? launch<false, 64, true>(p, stream) : launch<false, 128, true>(p, stream);
     return p.d == 64 ? launch<false, 64, false>(p, stream) : launch<false, 128, false>(p, stream);
 }
 
