@@ -901,6 +901,9 @@ int launch(const AttnParams& p, cudaStream_t stream) {
         // The split blocks go first and release their dependents at once, and the main launch
         // is allowed to start while they run (programmatic dependent launch): the two grids
         // are independent, so the SMs the short split CTAs leave go straight to main CTAs.
+        // The combine kernel is an ordinary launch behind both.  (All split CTAs are resident
+        // before the first main CTA starts, and each walks at most half the keys a main CTA
+        // walks, so the split grid is also the first to finish.)
         kern_split<<<(unsigned)(units * a.splits), kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test,
                                                                                       mk, mv, a);
         count_launch();
