@@ -199,6 +199,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C3")
+    ap.add_argument("--rows", type=int, nargs=2, metavar=("N_TRAIN", "N_TEST"), default=None,
+                    help="run the named workload's recipe at this many train / test rows (profiling on small cases)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-rows", type=int, default=96, help="oracle sample: query rows per head and call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -209,6 +211,8 @@ def main():
 
     from paper_2609_13031_b200 import workloads as W
     w = W.CONFIGS[args.workload]
+    if args.rows is not None:
+        w = w.scaled(args.rows[0], args.rows[1])
     if args.impl == "reference":
         run_reference(args, w)
         return
