@@ -10,7 +10,7 @@
 // Q K^T and P V are issued from different warps because a single warp cannot
 // issue tcgen05 instructions of this size fast enough to keep the tensor core fed.
 // A share of the exponentials (Cfg::kPolyPer16 pairs of every 16) is computed by a
-// polynomial on the FMA pipe instead of the MUFU; FP8ATTN_POLY16 overrides it at build time.
+// polynomial on the FMA pipe instead of the MUFU.
 // Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
 // thread pulls its whole score row into registers, releases S at once so that
 // the next Q K^T of its tile can run underneath the softmax, and writes the
@@ -87,11 +87,7 @@ struct Cfg {
     static constexpr int kPBufs = (kFp8 && kD == 64) ? 2 : 1;
     static constexpr bool kLateRescale = kD == 128;             // O rescale at the end of the step
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
-#ifdef FP8ATTN_POLY16
-    static constexpr int kPolyPer16 = FP8ATTN_POLY16;
-#else
     static constexpr int kPolyPer16 = kFp8 ? 4 : (kD == 128 ? 8 : 2);
-#endif
     static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= (kD == 128 ? 32 : 64)), "TMEM layout");
     static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
     static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
@@ -268,20 +264,6 @@ __device__ __forceinline__ void setmaxnreg_dec() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
 }
 
-#ifdef FP8ATTN_TRACE
-// Debug build only: clock stamps of CTA 0 (one lane per role) for a few steps.
-__device__ long long* g_trace_buf;
-#define FP8ATTN_TRACE_INIT() long long* const trace_buf = (blockIdx.x == 0) ? g_trace_buf : nullptr
-#define FP8ATTN_STAMP(slot, j)                                                         \
-    do {                                                                               \
-        if (trace_buf != nullptr && lane == 0 && (warp >= kSoftmaxWarps || (warp & 3) == 0) && (j) >= 64 && (j) < 80)                \
-            trace_buf[((j) - 64) * 32 + (slot)] = clock64();                           \
-    } while (0)
-#else
-#define FP8ATTN_TRACE_INIT() do { } while (0)
-#define FP8ATTN_STAMP(slot, j) do { } while (0)
-#endif
-
 // tcgen05.ld / wait / st of kCols consecutive columns (multiple of 16) in as few
 // instructions as possible
 template <int kCols>
@@ -343,6 +325,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t sticky_status;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -375,7 +358,11 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
 
     // A device error recorded earlier (and not yet read back by the host) is sticky:
     // nothing runs until fp8attn_last_device_status() has cleared it.
-    if (*reinterpret_cast<volatile uint32_t*>(args.status) != 0u) return;
+    // One thread reads it for the whole CTA, so that either every warp leaves or none does
+    // (a warp that left alone would leave the others blocked on the named barriers).
+    if (threadIdx.x == 0) sticky_status = *reinterpret_cast<volatile uint32_t*>(args.status);
+    __syncthreads();
+    if (sticky_status != 0u) return;
 
     // ---- set-up ----
     if (threadIdx.x == 0) {
@@ -407,7 +394,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     tc_fence_after_sync();
     const uint32_t tmem = __shfl_sync(0xffffffffu, tmem_slot, 0);
     Waiter w{args.status, false};
-    FP8ATTN_TRACE_INIT();
 
     if (warp == kTmaWarp) {
         setmaxnreg_dec<kRegsOther>();
@@ -490,7 +476,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 if (C::kSepP) named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
                 else w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
                 tc_fence_after_sync();
-                FP8ATTN_STAMP(20 + t, j);
                 issue_qk(t, sk);
             }
             if (elect_one()) mma_commit(smem_u32(&bars.k_empty[sk]));
@@ -509,7 +494,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
                 named_barrier_sync(kPFullBarrier0 + t, kSignalThreads);
                 tc_fence_after_sync();
-                FP8ATTN_STAMP(16 + t * 2, j);
                 if (elect_one()) {
                     const uint64_t b0 = dV + (uint64_t)((sv * C::kKVTileBytes) >> 4);
 #pragma unroll
@@ -524,7 +508,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     if (j + 1 == nkv) mma_commit(smem_u32(&bars.o_full[t]));
                 }
                 __syncwarp();
-                FP8ATTN_STAMP(17 + t * 2, j);
             }
         }
     } else {
@@ -552,7 +535,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             for (int j = 0; j < nkv; ++j) {
                 w.wait(smem_u32(&bars.s_full[t]), j & 1, kWaitSFull);
                 tc_fence_after_sync();
-                FP8ATTN_STAMP(t * 8 + 0, j);
                 // ---- the whole score row of this thread into registers ----
                 uint32_t s[kKeys];
                 tmem_ld_cols<kKeys>(tS, s);
@@ -562,7 +544,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     tc_fence_before_sync();
                     named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
                 }
-                FP8ATTN_STAMP(t * 8 + 1, j);
                 const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)(j0 + j) * kKeys);
                 if (valid < kKeys) {
 #pragma unroll
@@ -599,7 +580,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 const bool rescale = j > 0 && __any_sync(0xffffffffu, m_new > m);
                 float f = 1.0f;
                 if (rescale) {
-                    FP8ATTN_STAMP(t * 8 + 7, j);
                     f = ex2((m - m_new) * c);
                     const uint64_t ff = pack2(f, f);
                     l2a = mul2(l2a, ff);
@@ -624,7 +604,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 m = m_new;
                 const float nb = lift - m * c;
                 const uint64_t nbnb = pack2(nb, nb);
-                FP8ATTN_STAMP(t * 8 + 2, j);
                 // ---- p = 2^(c*s - c*m + lift), row sums, P tile into tensor memory ----
 #pragma unroll
                 for (int k0 = 0; k0 < kKeys; k0 += 32) {
@@ -664,15 +643,12 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         }
                     }
                     if (C::kPBufs == 1 && k0 == 0 && !pv_done) {
-                        FP8ATTN_STAMP(t * 8 + 5, j);
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
                         pv_done = true;
-                        FP8ATTN_STAMP(t * 8 + 6, j);
                     }
                     tmem_st_cols<kPPer32>(tP + (uint32_t)((C::kPBufs == 2 ? (j & 1) * C::kPCols : 0) + (k0 / 32) * kPPer32), p);
                 }
-                FP8ATTN_STAMP(t * 8 + 3, j);
                 if (C::kPBufs == 2 && !pv_done) {
                     // P V of the previous step has had this whole step to finish; once it
                     // has, the buffer that the NEXT step writes (the one it read) is free.
@@ -700,7 +676,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 tmem_wait_st();
                 tc_fence_before_sync();
                 named_barrier_arrive(kPFullBarrier0 + t, kSignalThreads);
-                FP8ATTN_STAMP(t * 8 + 4, j);
             }
             // ---- row sum ----
             float l;
@@ -766,6 +741,10 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
     }
     // ---- teardown ----
+    // Launched behind the split grid with programmatic stream serialization, this grid
+    // completes only after that one has (and its writes are visible): the combine kernel,
+    // ordered behind this grid, may then read the split grid's partial results.
+    if (!kSplit) asm volatile("griddepcontrol.wait;" ::: "memory");
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
@@ -887,25 +866,23 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     }
     auto kern = icl_attention_kernel<kFp8, kD, kHalf, false>;
     auto kern_split = icl_attention_kernel<kFp8, kD, kHalf, true>;
-    // the opt-in to large dynamic shared memory is per device (and per instantiation)
-    static bool attr_set[64] = {};
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)C::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(kern_split, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)C::kSmemBytes) != cudaSuccess)
-            return FP8ATTN_ERR_CUDA;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    // The opt-in to large dynamic shared memory is per device and per context; it is set on
+    // every call (a cached flag would go stale when the context is destroyed).
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes) !=
+            cudaSuccess ||
+        (units > 0 && cudaFuncSetAttribute(kern_split, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)C::kSmemBytes) != cudaSuccess))
+        return FP8ATTN_ERR_CUDA;
     if (units > 0) {
         // The split blocks go first and release their dependents at once, and the main launch
         // is allowed to start while they run (programmatic dependent launch): the two grids
         // are independent, so the SMs the short split CTAs leave go straight to main CTAs.
-        // The combine kernel is an ordinary launch behind both.  (All split CTAs are resident
-        // before the first main CTA starts, and each walks at most half the keys a main CTA
-        // walks, so the split grid is also the first to finish.)
+        // The combine kernel is an ordinary launch behind the main grid, and the main grid
+        // executes griddepcontrol.wait before it exits, so its completion implies that of the
+        // split grid and the visibility of the partial results.
         kern_split<<<(unsigned)(units * a.splits), kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test,
                                                                                       mk, mv, a);
+        if (cudaGetLastError() != cudaSuccess) return FP8ATTN_ERR_CUDA;
         count_launch();
     }
     if (a.full_blocks > 0) {
@@ -947,15 +924,6 @@ __global__ void wait_timeout_selftest_kernel(uint32_t* status, uint64_t limit_ns
     Waiter w{status, false, limit_ns};
     w.wait(smem_u32(&bar), 0, kWaitSelfTest);
 }
-
-#ifdef FP8ATTN_TRACE
-// Debug build only: where the kernels of CTA 0 write their clock stamps
-// (16 steps x 32 slots of int64), or NULL to switch tracing off.
-extern "C" int fp8attn_debug_set_trace(void* device_buffer) {
-    long long* p = static_cast<long long*>(device_buffer);
-    return cudaMemcpyToSymbol(g_trace_buf, &p, sizeof(p)) == cudaSuccess ? 0 : 4;
-}
-#endif
 
 int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream) {
     wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
