@@ -27,10 +27,30 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from an ncu capture of the
-# same workload (summaries under profiles/); None where no capture exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"C3": 219.0e6 + 136.6e6}
 NOMINAL_FP8_OVER_BF16 = 2.0           # dense tensor peak ratio (4.5 / 2.25 PFLOP/s)
+# exponentials per clock per SM: the 16-lane MUFU alone, and with a quarter of them on the FMA pipe
+SOFTMAX_MUFU_PER_CLK_SM = 16.0
+SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM = 16.0 / 0.75
+
+
+def ncu_dram_traffic(workload: str):
+    """DRAM bytes of one attention launch (dram__bytes_read.sum + dram__bytes_write.sum) from
+    the ncu capture recorded under profiles/ for this workload, with the commit it was taken
+    at; None where no capture exists."""
+    path = os.path.join(ROOT, "profiles", f"icl_attention_fp8_{workload}_dram_traffic.txt")
+    try:
+        kv = {}
+        with open(path) as f:
+            for ln in f:
+                if "=" in ln and not ln.lstrip().startswith("#"):
+                    k, v = ln.split("=", 1)
+                    kv[k.strip()] = v.strip()
+        return {"bytes": float(kv["dram_bytes_read"]) + float(kv["dram_bytes_write"]),
+                "captured_at_commit": kv.get("commit"), "launch": kv.get("launch")}
+    except Exception:
+        return None
+
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -45,7 +65,7 @@ def load_peaks():
 
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU while the timed region runs
-    (one streaming ``nvidia-smi -lms 100`` child, read line by line)."""
+    (one streaming ``nvidia-smi -lms 20`` child, read line by line)."""
 
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -58,7 +78,7 @@ class ClockSampler(threading.Thread):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -77,14 +97,21 @@ class ClockSampler(threading.Thread):
                 if val.lower().startswith("active"):
                     self.reasons.add(name)
 
-    def result(self):
+    def restart(self):
+        """Forget the samples so far (the next ones belong to a new region)."""
+        self.sm = []
+        self.reasons = set()
+
+    def snapshot(self):
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.sm)), "sm_min_mhz": float(np.min(self.sm)),
+                "sm_max_mhz": self.max_sm, "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+    def stop(self):
         if self.proc is not None:
             self.proc.terminate()          # our own child, by handle
             self.join(timeout=10)
-        if not self.sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
-        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_sm,
-                "reasons": sorted(self.reasons), "samples": len(self.sm)}
 
 
 def library_fp8_gemm_rate(seconds: float = 3.0, n: int = 8192):
@@ -206,6 +233,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-bf16", action="store_true")
     ap.add_argument("--no-fp8-gemm", action="store_true", help="skip the library FP8 GEMM rate (context figure)")
+    ap.add_argument("--preroll", type=float, default=3.0,
+                    help="seconds of untimed steps under the same load before each timed region, so that the "
+                         "timed steps run at the clock the board's power limit settles on")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -294,16 +324,29 @@ def main():
         raise RuntimeError(f"device status {status}")
     sampler = ClockSampler(local)
     sampler.start()
-    # keep the GPU busy (untimed) until the sampler delivers, so every sample is under load
-    for _ in range(200):
+
+    def preroll(step_fn):
+        """Untimed steps under the same load for at least --preroll seconds (at least one step):
+        the timed steps then run at the clock that the power limit settles on, the state the
+        sustained roofline denominator was measured in."""
+        t0 = time.perf_counter()
+        n = 0
+        while True:
+            step_fn()
+            n += 1
+            if n % 4 == 0 or n == 1:
+                torch.cuda.synchronize()
+                if time.perf_counter() - t0 >= args.preroll:
+                    break
+        torch.cuda.synchronize()
+        return n, time.perf_counter() - t0
+
+    def fp8_step():
         quantize_all()
         attention_fp8()
-        torch.cuda.synchronize()
-        if sampler.sm:
-            break
-    preroll = (list(sampler.sm), set(sampler.reasons))
-    sampler.sm.clear()
-    sampler.reasons.clear()
+
+    pre_n, pre_s = preroll(fp8_step)
+    sampler.restart()
     launches0 = api.launch_count()
     marks = []
     sync_all()
@@ -320,31 +363,35 @@ def main():
     e_end.record()
     sync_all()
     launches = api.launch_count() - launches0
-    if not sampler.sm:                      # timed region shorter than one sampling period:
-        sampler.sm, sampler.reasons = preroll   # the samples of the untimed pre-roll under the same load
-    clocks = sampler.result()
+    clocks = sampler.snapshot()
+    clocks["preroll_seconds"] = pre_s
     total_ms = max_over_ranks(e_start.elapsed_time(e_end))
     ms_step = total_ms / args.steps
-    ms_quant = float(np.mean([a.elapsed_time(b) for a, b, _ in marks]))
-    ms_attn = float(np.mean([b.elapsed_time(c) for _, b, c in marks]))
+    t_quant = np.array([a.elapsed_time(b) for a, b, _ in marks])
+    t_attn = np.array([b.elapsed_time(c) for _, b, c in marks])
+    ms_quant, ms_attn = float(np.mean(t_quant)), float(np.mean(t_attn))
     status = api.last_device_status(ws)
     if status != (0, 0):
         raise RuntimeError(f"device status {status}")
 
-    # ---- the in-build BF16 path on the same inputs ----
-    ms_bf16 = None
+    # ---- the in-build BF16 path on the same inputs: same pre-roll, same number of launches ----
+    ms_bf16, t_bf16, clocks_bf16 = None, None, None
     if not args.no_bf16:
-        for _ in range(2):
-            attention_bf16()
+        preroll(attention_bf16)
+        sampler.restart()
         sync_all()
-        a, b = ev(), ev()
-        n_bf = max(2, min(args.steps, 5))
-        a.record()
-        for _ in range(n_bf):
+        bmarks = []
+        for _ in range(args.steps):
+            a, b = ev(), ev()
+            a.record()
             attention_bf16()
-        b.record()
+            b.record()
+            bmarks.append((a, b))
         sync_all()
-        ms_bf16 = max_over_ranks(a.elapsed_time(b)) / n_bf
+        clocks_bf16 = sampler.snapshot()
+        t_bf16 = np.array([a.elapsed_time(b) for a, b in bmarks])
+        ms_bf16 = max_over_ranks(float(np.mean(t_bf16)))
+    sampler.stop()
 
     # ---- end to end: pinned host inputs -> device -> path -> host outputs, every step ----
     # Every step copies its own inputs from pinned host memory and its own results back.  The
@@ -411,6 +458,21 @@ def main():
     h2d = sum(t.numel() * t.element_size() for t in host.values())
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
 
+    # ---- one call, host to host, nothing overlapped: copy in, quantize, attention, copy out ----
+    single = []
+    for _ in range(max(3, min(args.steps, 5))):
+        sync_all()
+        t0 = time.perf_counter()
+        for k in host:
+            dev[k].copy_(host[k], non_blocking=True)
+        quantize_all()
+        attention_fp8()
+        host_out["o_tr"].copy_(buf["o_tr"], non_blocking=True)
+        host_out["o_te"].copy_(buf["o_te"], non_blocking=True)
+        torch.cuda.synchronize()
+        single.append(1e3 * (time.perf_counter() - t0))
+    ms_single = max_over_ranks(float(np.median(single)))
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -427,11 +489,27 @@ def main():
 
     if rank == 0:
         flops = w.flops
-        tf_step = world * flops / (ms_step * 1e-3) / 1e12
-        tf_attn = flops / (ms_attn * 1e-3) / 1e12
+        tf = lambda ms: flops / (ms * 1e-3) / 1e12
+        tf_step = world * tf(ms_step)
+        tf_attn = tf(ms_attn)
         peak_fp8 = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops_sustained"]
         peak_fp8_burst = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops"]
         quant_bytes = w.B * w.H * w.d * (5 * 3 * w.n_train + 3 * w.n_test)
+        # secondary roofline: the exponential path.  One exponential per score; the MUFU
+        # evaluates 16 per clock per SM, and with a quarter of them on the FMA pipe the
+        # limit is 21.3.  Clock = the median SM clock sampled during the timed steps.
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        scores = float(w.B) * w.H * w.n_train * (w.n_train + w.n_test)
+        softmax = None
+        if clocks.get("sm_mhz"):
+            per_clk_sm = scores / (ms_attn * 1e-3) / (sms * clocks["sm_mhz"] * 1e6)
+            softmax = {"scores_per_clk_per_sm": per_clk_sm,
+                       "mufu_only_peak": SOFTMAX_MUFU_PER_CLK_SM,
+                       "frac_of_mufu_only": per_clk_sm / SOFTMAX_MUFU_PER_CLK_SM,
+                       "quarter_on_fma_peak": SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM,
+                       "frac": per_clk_sm / SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM,
+                       "clock_mhz": clocks["sm_mhz"], "sms": sms}
+        traffic = ncu_dram_traffic(w.name)
         line = {
             "metric": "fp8_icl_attention_tflops", "value": tf_step, "unit": "TFLOP/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
@@ -440,17 +518,27 @@ def main():
             "config": {"workload": workload_label(w),
                        "step": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
                        "l2": "inputs larger than L2 (bf16 inputs %.0f MB)" % (h2d / 1e6),
+                       "preroll": "%d untimed steps (%.1f s) under the same load before the timed steps" % (pre_n, pre_s),
                        "replicas": world},
             "clocks": clocks,
-            "e2e": {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+            "e2e": {"value": world * tf(ms_e2e), "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
+                    "kind": "pipelined throughput: copies of neighbouring steps overlap the compute (3 streams, 2 buffer sets)",
+                    "single_call_ms": ms_single, "single_call_value": world * tf(ms_single),
+                    "single_call_kind": "median host-to-host latency of one step, nothing overlapped"},
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "kernel": "icl_attention_kernel<fp8>",
                          "achieved": tf_attn, "peak": peak_fp8, "unit": "TFLOP/s",
-                         "frac": tf_attn / peak_fp8, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
-                         "peak_source": f"2 x bf16_tflops_sustained ({peak_kind}), nominal fp8:bf16 ratio",
+                         "frac": tf_attn / peak_fp8,
+                         "achieved_median": tf(float(np.median(t_attn))),
+                         "achieved_best": tf(float(np.min(t_attn))),
+                         "traffic": None if traffic is None else traffic["bytes"],
+                         "traffic_source": traffic,
+                         "peak_source": f"2 x bf16_tflops_sustained ({peak_kind}), nominal fp8:bf16 ratio; the timed "
+                                        "steps follow a pre-roll under load, i.e. the sustained clock state",
                          "frac_of_burst_peak": tf_attn / peak_fp8_burst,
                          "frac_of_nominal_4500": tf_attn / 4500.0,
+                         "softmax": softmax,
                          "library_fp8_gemm_tflops": None if not isinstance(fp8_gemm, tuple) else
                          {"burst": fp8_gemm[0], "sustained": fp8_gemm[1],
                           "how": "torch._scaled_mm e4m3 8192^3, best of 10 / back to back for 3 s, same run"},
@@ -460,8 +548,13 @@ def main():
             "cpu_baseline": cpu_baseline,
             "breakdown": {
                 "ms_quantize": ms_quant, "ms_attention_fp8": ms_attn, "ms_attention_bf16": ms_bf16,
+                "ms_attention_fp8_median": float(np.median(t_attn)), "ms_attention_fp8_best": float(np.min(t_attn)),
+                "ms_attention_bf16_median": None if t_bf16 is None else float(np.median(t_bf16)),
+                "ms_attention_bf16_best": None if t_bf16 is None else float(np.min(t_bf16)),
+                "ms_quantize_median": float(np.median(t_quant)), "ms_quantize_best": float(np.min(t_quant)),
+                "clocks_bf16": clocks_bf16,
                 "attention_fp8_tflops": tf_attn,
-                "attention_bf16_tflops": None if ms_bf16 is None else flops / (ms_bf16 * 1e-3) / 1e12,
+                "attention_bf16_tflops": None if ms_bf16 is None else tf(ms_bf16),
                 "speedup_vs_bf16_attention_only": None if ms_bf16 is None else ms_bf16 / ms_attn,
                 "speedup_vs_bf16_with_quantize": None if ms_bf16 is None else ms_bf16 / (ms_attn + ms_quant),
                 "quantize_gbs": quant_bytes / (ms_quant * 1e-3) / 1e9,

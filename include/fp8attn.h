@@ -74,12 +74,20 @@ int fp8attn_quantize_ex(const void* x_16bit, int B, int H, int64_t rows, int d,
                         const float* scale_in, void* x_fp8, float* scale_out, uint32_t flags,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* The four quantizations of one ICL attention call in two launches instead of
- * seven (same arithmetic and bit-identical results to four fp8attn_quantize
- * calls): per-head absmax scales for Q_train, K and V (paper Eq. 2), and Q_test
- * quantized with the train-query scale (Method section, shared query scale).  It
- * removes most of the launch overhead that makes quantization dominate at small
- * train-row counts (the paper's latency tables below ~8k rows).
+/* The four quantizations of one ICL attention call in one or two launches
+ * instead of seven (same arithmetic and bit-identical results to four
+ * fp8attn_quantize calls): per-head absmax scales for Q_train, K and V (paper
+ * Eq. 2), and Q_test quantized with the train-query scale (Method section, shared
+ * query scale).  It removes most of the launch overhead that makes quantization
+ * dominate at small train-row counts (the paper's latency tables below ~8k rows).
+ * A call whose 16-bit inputs total at most 48 MB (they stay in L2) runs as ONE
+ * launch of at most two thread blocks per SM: maximum, a grid-wide arrival
+ * counter, conversion.  The blocks wait for one another, which presumes that they
+ * are all resident at once, as they are on a GPU that runs nothing else; the wait
+ * is bounded (2 s) and ends in FP8ATTN_ERR_TIMEOUT in the workspace's status word.
+ * Callers that share the GPU with long-running kernels of other streams can ask
+ * for the two-launch form with FP8ATTN_QKV_TWO_LAUNCHES (the _ex call).  Larger
+ * calls always take two launches (maximum; conversion).
  *
  *   q_train, k, v   in  bf16 [B,H,n_train,d]      q_test in bf16 [B,H,n_test,d] (NULL iff n_test == 0)
  *   *_fp8           out e4m3, same shapes          scale_q/k/v out fp32 [B,H]
@@ -105,9 +113,11 @@ int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, cons
  * and V (the paper's method section notes that the quantization overhead is what
  * limits small tables).  No maximum pass runs: one launch, each element read
  * once; values outside a given scale's range saturate at +-448.  Not combinable
- * with FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS. */
+ * with FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS.
+ * FP8ATTN_QKV_TWO_LAUNCHES: never take the one-launch path of small calls. */
 #define FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS 1u
 #define FP8ATTN_SCALES_GIVEN 4u
+#define FP8ATTN_QKV_TWO_LAUNCHES 8u
 int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test,
                             int B, int H, int64_t n_train, int64_t n_test, int d,
                             void* q_train_fp8, void* k_fp8, void* v_fp8, void* q_test_fp8,
@@ -154,8 +164,8 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
 /* Variants of the two forward calls with a flags word.
  *
  * FP8ATTN_TEST_ROWS_USE_KV_HEAD0: grouped-query test->train attention as in
- * TabPFN-v3 (paper appendix, noise-experiment details: "test rows attend to the
- * first K,V head"): the test queries of every head h of a table attend to the
+ * TabPFN-v3 (paper appendix, noise-experiment details, where the test->train call
+ * uses K/V head 0 only): the test queries of every head h of a table attend to the
  * keys and values of head 0 of that table (and use head 0's K and V scales; the
  * query scale stays head h's train-query scale).  Train rows are unaffected.
  * K and V are still passed, and were quantized, as full [B,H,n_train,d] tensors,
@@ -226,9 +236,11 @@ int fp8attn_gate_use_fp8(int64_t n_train);
  *
  *   x_bf16 in bf16 [B,H,rows,d]; out_bf16 out, same shape (may alias x_bf16);
  *   rho_out out fp32 [B,H] or NULL.
- * Z is a pure function of (seed, stream_id, b*H+h, element index): a run is
- * reproducible from the seed, and different stream_id values (one per tensor and
- * layer, say) give independent fields.  Perturbing K and V once and passing the
+ * Z is a pure function of (seed, stream_id, b*H+h, element index): the noise
+ * field is reproducible from the seed, and different stream_id values (one per
+ * tensor and layer, say) give independent fields.  rho is summed with fp64 atomic
+ * additions whose order varies between runs, so rho can differ in its last bit from
+ * run to run, and with it (rarely) the rounding of an output element.  Perturbing K and V once and passing the
  * result to fp8attn_icl_forward / bf16attn_icl_forward is the paper's
  * "coordinated" arm: both attention calls then consume the same noisy K, V.
  * The normals come from Box-Muller in fp32 (hardware log / sin / cos), the sum of

@@ -30,6 +30,7 @@ EXPORTS = (
 QUERY_SCALE_FROM_ALL_ROWS = 1
 INPUT_FP16 = 2
 SCALES_GIVEN = 4
+QKV_TWO_LAUNCHES = 8
 # flags of fp8attn_icl_forward_ex / bf16attn_icl_forward_ex
 TEST_ROWS_USE_KV_HEAD0 = 1
 TEST_ROWS_ONLY = 2

@@ -9,6 +9,17 @@ namespace fp8attn {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+size_t split_scratch_bytes(int d) {
+    // one unit per SM at most; without a device to ask (size queries on a host without
+    // a GPU) the size assumes the largest sm_100 part
+    constexpr int kSmsWithoutDevice = 160;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = kSmsWithoutDevice;
+    return (size_t)sms * 256 * (size_t)(d + 4) * sizeof(float);
+}
+
 namespace {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -118,7 +129,8 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS | FP8ATTN_INPUT_FP16 | FP8ATTN_SCALES_GIVEN))
+    if (flags & ~(uint32_t)(FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS | FP8ATTN_INPUT_FP16 | FP8ATTN_SCALES_GIVEN |
+                            FP8ATTN_QKV_TWO_LAUNCHES))
         return FP8ATTN_ERR_INVALID_ARG;
     if ((flags & FP8ATTN_SCALES_GIVEN) && (flags & FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS))
         return FP8ATTN_ERR_INVALID_ARG;
@@ -133,9 +145,13 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
     rc = check_device();
     if (rc != FP8ATTN_OK) return rc;
     uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
+    char* ws = static_cast<char*>(workspace);
     return launch_quantize_qkv(q_train, k, v, q_test, (int64_t)B * H, n_train * (int64_t)d,
                                n_test * (int64_t)d, q_train_fp8, k_fp8, v_fp8, q_test_fp8, scale_q, scale_k,
-                               scale_v, amax, flags, static_cast<cudaStream_t>(cuda_stream));
+                               scale_v, amax, flags, reinterpret_cast<uint32_t*>(ws + kWsStatusOffset),
+                               reinterpret_cast<uint32_t*>(ws + kWsCounterOffset),
+                               reinterpret_cast<float*>(ws + ws_partial_offset(B, H)),
+                               static_cast<cudaStream_t>(cuda_stream));
 }
 
 int fp8attn_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test, int B,
@@ -230,7 +246,9 @@ int fp8attn_last_device_status(void* workspace, void* cuda_stream, uint32_t* det
     if (cudaMemcpy(words, workspace, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess)
         return FP8ATTN_ERR_CUDA;
     if (detail) *detail = words[1];
-    if (words[0] != 0 && cudaMemset(workspace, 0, sizeof(words)) != cudaSuccess) return FP8ATTN_ERR_CUDA;
+    // after an error: clear the status words, and the arrival counters a one-launch
+    // quantization that gave up may have left behind
+    if (words[0] != 0 && cudaMemset(workspace, 0, kWsAmaxOffset) != cudaSuccess) return FP8ATTN_ERR_CUDA;
     return (int)words[0];
 }
 

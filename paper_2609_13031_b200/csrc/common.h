@@ -15,18 +15,30 @@ namespace fp8attn {
 //                       patterns): one is used by fp8attn_quantize, all three (Q, K, V)
 //                       by fp8attn_quantize_qkv; cleared at the start of every call.
 //                       fp8attn_perturb keeps its per-head sums of squares (fp64) here too.
+//   [16,24)  the two grid-wide arrival counters of the one-launch quantizer; zero between calls
+//   after the accumulators: partial maxima of the one-launch quantizer, one fp32 per
+//                       (block, head segment) pair: kOneLaunchMaxBlocks + 4*B*H slots
 constexpr size_t kWsStatusOffset = 0;
 constexpr size_t kWsDetailOffset = 4;
+constexpr size_t kWsCounterOffset = 16;
 constexpr size_t kWsAmaxOffset = 256;
+constexpr int kOneLaunchMaxBlocks = 1024;
+// detail code (bits 24..31 of the detail word) of an expired wait at the one-launch quantizer's grid barrier
+constexpr uint32_t kDetailQuantizeGridWait = 32;
 
-inline size_t workspace_bytes(int B, int H) {
+inline size_t ws_amax_bytes(int B, int H) {
     size_t amax = (size_t)12 * (size_t)B * (size_t)H;
-    return kWsAmaxOffset + ((amax + 255) / 256) * 256;
+    return ((amax + 255) / 256) * 256;
+}
+inline size_t ws_partial_offset(int B, int H) { return kWsAmaxOffset + ws_amax_bytes(B, H); }
+inline size_t workspace_bytes(int B, int H) {
+    size_t partial = sizeof(float) * ((size_t)kOneLaunchMaxBlocks + (size_t)4 * (size_t)B * (size_t)H);
+    return ws_partial_offset(B, H) + ((partial + 255) / 256) * 256;
 }
 
 // Scratch of the tail split (FP8ATTN_SPLIT_TAIL), appended to the workspace: partial results
-// of fewer than one CTA per SM, 256 rows of d + 4 floats each; sized for up to 192 SMs.
-inline size_t split_scratch_bytes(int d) { return (size_t)192 * 256 * (size_t)(d + 4) * sizeof(float); }
+// of fewer than one CTA per SM of the current device, 256 rows of d + 4 floats each (api.cu).
+size_t split_scratch_bytes(int d);
 
 void count_launch();
 
@@ -35,10 +47,13 @@ int launch_quantize(const void* x_bf16, int64_t n_heads, int64_t elems_per_head,
                     const float* scale_in, void* x_fp8, float* scale_out,
                     uint32_t* amax_bits, uint32_t flags, cudaStream_t stream);
 
+// `status`, `counters`, `partial`: the workspace's status words, arrival counters and
+// partial-maximum slots (the one-launch path for small calls uses them).
 int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const void* q_test,
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
-                        float* scale_v, uint32_t* amax_bits, uint32_t flags, cudaStream_t stream);
+                        float* scale_v, uint32_t* amax_bits, uint32_t flags, uint32_t* status,
+                        uint32_t* counters, float* partial, cudaStream_t stream);
 
 // perturb.cu
 int launch_perturb(const void* x_bf16, int64_t n_heads, int64_t elems_per_head, float epsilon,

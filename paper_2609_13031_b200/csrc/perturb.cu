@@ -78,9 +78,11 @@ __device__ __forceinline__ uint32_t perturb_word(uint32_t w, uint64_t key, int64
     return packed;
 }
 
+// x and out may be the same buffer (each vector is read, then written, by one thread), so
+// neither is __restrict__ and x is read with ordinary coherent loads.
 __global__ void __launch_bounds__(kThreads)
-perturb_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, const double* __restrict__ sumsq,
-               float epsilon, uint64_t seed, uint32_t stream_id, uint4* __restrict__ out,
+perturb_kernel(const uint4* x, int64_t vecs_per_head, const double* __restrict__ sumsq,
+               float epsilon, uint64_t seed, uint32_t stream_id, uint4* out,
                float* __restrict__ rho_out) {
     const int64_t head = blockIdx.y;
     const float rho = (float)sqrt(sumsq[head] / (double)(vecs_per_head * 8));
@@ -91,7 +93,7 @@ perturb_kernel(const uint4* __restrict__ x, int64_t vecs_per_head, const double*
     uint4* oh = out + head * vecs_per_head;
     for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < vecs_per_head;
          i += (int64_t)gridDim.x * kThreads) {
-        const uint4 v = ld_nc_v4(xh + i);
+        const uint4 v = xh[i];
         uint4 o;
         o.x = perturb_word(v.x, key, 4 * i + 0, amp);
         o.y = perturb_word(v.y, key, 4 * i + 1, amp);
@@ -109,7 +111,11 @@ int launch_perturb(const void* x_bf16, int64_t n_heads, int64_t elems_per_head, 
     if (n_heads <= 0 || elems_per_head <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     const int64_t vecs = elems_per_head / 8;
-    int64_t want = (148 * 16 + n_heads - 1) / n_heads, have = (vecs + kThreads - 1) / kThreads;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return FP8ATTN_ERR_CUDA;
+    int64_t want = ((int64_t)sms * 16 + n_heads - 1) / n_heads, have = (vecs + kThreads - 1) / kThreads;
     const unsigned bx = (unsigned)(want < have ? (want < 1 ? 1 : want) : (have < 1 ? 1 : have));
     if (cudaMemsetAsync(sumsq, 0, sizeof(double) * n_heads, stream) != cudaSuccess) return FP8ATTN_ERR_CUDA;
     sumsq_kernel<<<dim3(bx, (unsigned)n_heads), kThreads, 0, stream>>>((const uint4*)x_bf16, vecs, sumsq);

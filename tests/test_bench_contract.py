@@ -35,7 +35,7 @@ def test_gpu_arm_line():
     assert COMMON | {"clocks", "gpu_launches", "roofline"} <= set(d)
     assert d["n_gpus"] == 1 and d["steps"] == 4 and d["warmup"] >= 3 and d["scaling"] == "weak"
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["dtype"] == "fp8_e4m3" and d["data"] == "synthetic"
-    assert d["gpu_launches"] >= 3 * d["steps"]
+    assert d["gpu_launches"] >= 2 * d["steps"]      # one-launch quantizer + attention on a small table
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and d["e2e"]["value"] > 0

@@ -46,7 +46,7 @@ def test_step_replays_from_a_cuda_graph():
     with torch.cuda.graph(graph):
         step()
     per_step = api.launch_count() - launches
-    assert per_step == 3                                   # absmax, convert, attention
+    assert per_step == 2                                   # one-launch quantizer, attention
 
     for data, (w_tr, w_te, w_sq) in zip((first, second), want):
         for k in x:

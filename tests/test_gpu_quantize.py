@@ -114,32 +114,56 @@ def test_argument_errors_are_reported_on_the_host():
 @pytest.mark.parametrize("cfg,n,m", [("C1", 512, 128), ("C2", 8192, 2048), ("C4", 3000, 0), ("C3", 4096, 1),
                                       ("C5", 1, 0)])
 def test_fused_qkv_quantize_matches_oracle(cfg, n, m):
-    """fp8attn_quantize_qkv (two launches) is bit-identical to the oracle, including the
-    shared train-query scale for the test queries."""
+    """fp8attn_quantize_qkv is bit-identical to the oracle, including the shared train-query
+    scale for the test queries: as one launch (these sizes are small calls), and as two launches
+    when asked for.  Twice in a row on one workspace: the one-launch path must leave its
+    counters clean."""
     w = W.CONFIGS[cfg].scaled(n, m)
     g = W.generate(w)
     ws = api.new_workspace(w.B, w.H)
-    o = api.quantize_qkv(to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]),
-                         to_dev(g["q_test"]) if m else None, ws)
     rq, rsq = oracle.quantize(g["q_train"])
     rk, rsk = oracle.quantize(g["k"])
     rv, rsv = oracle.quantize(g["v"])
-    for got, ref in ((o["q8"], rq), (o["k8"], rk), (o["v8"], rv), (o["sq"], rsq), (o["sk"], rsk), (o["sv"], rsv)):
-        assert np.array_equal(got.cpu().numpy(), ref)
-    if m:
-        rt, _ = oracle.quantize(g["q_test"], scale_in=rsq)
-        assert np.array_equal(o["t8"].cpu().numpy(), rt)
+    dev = [to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]), to_dev(g["q_test"]) if m else None]
+    for flags, launches in ((0, 1), (0, 1), (api.QKV_TWO_LAUNCHES, 2), (0, 1)):
+        before = api.launch_count()
+        o = api.quantize_qkv(*dev, ws, flags=flags)
+        assert api.launch_count() - before == launches
+        for got, ref in ((o["q8"], rq), (o["k8"], rk), (o["v8"], rv), (o["sq"], rsq), (o["sk"], rsk), (o["sv"], rsv)):
+            assert np.array_equal(got.cpu().numpy(), ref)
+        if m:
+            rt, _ = oracle.quantize(g["q_test"], scale_in=rsq)
+            assert np.array_equal(o["t8"].cpu().numpy(), rt)
+        assert api.last_device_status(ws) == (0, 0)
+
+
+def test_fused_qkv_large_call_takes_two_launches():
+    """Above the one-launch size (48 MB of 16-bit input) the call is a maximum pass and a
+    conversion pass; bit-identical to the oracle all the same."""
+    w = W.CONFIGS["C3"].scaled(20000, 3000)      # 8 heads x 128 x (3 x 20000 + 3000) x 2 B = 129 MB
+    g = W.generate(w)
+    ws = api.new_workspace(w.B, w.H)
+    before = api.launch_count()
+    o = api.quantize_qkv(to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]), to_dev(g["q_test"]), ws)
+    assert api.launch_count() - before == 2
+    rq, rsq = oracle.quantize(g["q_train"])
+    rt, _ = oracle.quantize(g["q_test"], scale_in=rsq)
+    rv, rsv = oracle.quantize(g["v"])
+    assert np.array_equal(o["q8"].cpu().numpy(), rq) and np.array_equal(o["t8"].cpu().numpy(), rt)
+    assert np.array_equal(o["v8"].cpu().numpy(), rv) and np.array_equal(o["sv"].cpu().numpy(), rsv)
     assert api.last_device_status(ws) == (0, 0)
 
 
-def test_fused_qkv_query_scale_from_all_rows():
-    """Single-call form: one query scale over train and test queries together."""
+@pytest.mark.parametrize("extra", [0, api.QKV_TWO_LAUNCHES])
+def test_fused_qkv_query_scale_from_all_rows(extra):
+    """Single-call form: one query scale over train and test queries together (one-launch and
+    two-launch paths)."""
     w = W.CONFIGS["C2"].scaled(700, 900)
     g = W.generate(w)
     g["q_test"] = f32_to_bf16_bits(W.bf16_bits_to_f32(g["q_test"]) * np.float32(3.0))   # test rows set the maximum
     ws = api.new_workspace(w.B, w.H)
     o = api.quantize_qkv(to_dev(g["q_train"]), to_dev(g["k"]), to_dev(g["v"]), to_dev(g["q_test"]), ws,
-                         flags=api.QUERY_SCALE_FROM_ALL_ROWS)
+                         flags=api.QUERY_SCALE_FROM_ALL_ROWS | extra)
     _, s_all = oracle.quantize(np.concatenate([g["q_train"], g["q_test"]], axis=2))
     rq, _ = oracle.quantize(g["q_train"], scale_in=s_all)
     rt, _ = oracle.quantize(g["q_test"], scale_in=s_all)

@@ -110,7 +110,7 @@ def test_quantize_fp16_input_is_bit_exact(cfg, n, m):
     t8, st = api.quantize(fp16_dev(g["q_test"]), ws, scale_in=sq)
     assert np.array_equal(q8.cpu().numpy(), ref[0]) and np.array_equal(sq.cpu().numpy(), ref[4])
     assert np.array_equal(t8.cpu().numpy(), ref[1]) and np.array_equal(st.cpu().numpy(), ref[4])
-    # ... and all four in two launches
+    # ... and all four in one call
     o = api.quantize_qkv(fp16_dev(g["q_train"]), fp16_dev(g["k"]), fp16_dev(g["v"]), fp16_dev(g["q_test"]), ws)
     for name, r in zip(("q8", "t8", "k8", "v8", "sq", "sk", "sv"), ref):
         assert np.array_equal(o[name].cpu().numpy(), r), name
