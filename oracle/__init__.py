@@ -131,6 +131,30 @@ def e4m3_decode_table() -> np.ndarray:
 _DTYPE16 = {"bf16": 0, "fp16": 1}
 
 
+def rounding_envelope(x: float) -> float:
+    """The oracle's worst-case e4m3 rounding error at magnitude x (the envelope behind Bnd)."""
+    lib = _load()
+    lib.oracle_rounding_envelope.restype = ctypes.c_double
+    lib.oracle_rounding_envelope.argtypes = [ctypes.c_double]
+    return float(lib.oracle_rounding_envelope(float(x)))
+
+
+def round_to_bf16(x: float) -> float:
+    """The oracle's fp32 -> nearest bf16 (as a float), used for the e4m3-P mode's output."""
+    lib = _load()
+    lib.oracle_round_to_bf16.restype = ctypes.c_float
+    lib.oracle_round_to_bf16.argtypes = [ctypes.c_float]
+    return float(lib.oracle_round_to_bf16(float(x)))
+
+
+def double_to_bf16_bits(v: float) -> int:
+    """The oracle's fp64 -> nearest bf16 bit pattern, used by the perturbation."""
+    lib = _load()
+    lib.oracle_double_to_bf16_bits.restype = ctypes.c_uint16
+    lib.oracle_double_to_bf16_bits.argtypes = [ctypes.c_double]
+    return int(lib.oracle_double_to_bf16_bits(float(v)))
+
+
 def half_to_float(bits: int) -> float:
     """Value of one IEEE fp16 bit pattern, by the format's definition."""
     return float(_load().oracle_half_to_float(int(bits) & 0xFFFF))

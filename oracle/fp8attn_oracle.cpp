@@ -171,6 +171,10 @@ void oracle_e4m3_encode_array(const float* y, int64_t n, uint8_t* out) {
 
 float oracle_half_to_float(uint16_t h) { return half_to_float(h); }
 
+// Exposed so that tests can pin them (no arithmetic of their own).
+double oracle_rounding_envelope(double x) { return rounding_envelope(x); }
+float oracle_round_to_bf16(float x) { return round_to_bf16(x); }
+
 // ---- quantize (Eq. 2) ------------------------------------------------------
 // x: bf16 (dtype16 = 0) or IEEE fp16 (dtype16 = 1) bit patterns [B,H,R,d] contiguous.
 // scale_in: NULL or [B*H] fp32.
@@ -380,6 +384,7 @@ static uint64_t perturb_mix64(uint64_t z) {
     return z ^ (z >> 31);
 }
 
+uint16_t oracle_double_to_bf16_bits(double v);
 static uint16_t double_to_bf16_bits(double v) {
     // nearest bf16 to v: the two bf16 neighbours of |v| are compared in fp64
     double a = std::fabs(v);
@@ -397,6 +402,8 @@ static uint16_t double_to_bf16_bits(double v) {
     uint32_t pick = dlo < dhi ? lo : (dhi < dlo ? hi : (((lo >> 16) & 1u) ? hi : lo));
     return (uint16_t)((pick >> 16) | (std::signbit(v) ? 0x8000u : 0u));
 }
+
+uint16_t oracle_double_to_bf16_bits(double v) { return double_to_bf16_bits(v); }
 
 void oracle_perturb(const uint16_t* x, int B, int H, int64_t R, int d, double eps, uint64_t seed,
                     uint32_t stream_id, uint16_t* out, double* rho_out, int nthreads) {

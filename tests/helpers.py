@@ -93,8 +93,39 @@ def check_bf16_attention(out, A, Abs, label="", rounding=2.0 ** -9):
 
 
 def sample_rows(n, count, seed):
-    """Query rows to check: tile boundaries, first/last, plus seeded random rows."""
+    """Query rows to check: the fixed tile-boundary rows (first two and last two CTAs of a
+    head), plus ``count`` seeded rows stratified over the whole row range -- one row drawn
+    in each of ``count`` equal strata, so that the middle query blocks of a large table are
+    hit as surely as its ends."""
     fixed = [r for r in (0, 1, 127, 128, 255, 256, 257, n - 129, n - 128, n - 2, n - 1) if 0 <= r < n]
     rng = np.random.default_rng(seed)
-    extra = rng.integers(0, n, size=max(0, count - len(fixed))) if n > 0 else []
-    return np.unique(np.array(list(fixed) + list(extra), dtype=np.int64))
+    extra = []
+    if n > 0 and count > 0:
+        edges = np.linspace(0, n, count + 1).astype(np.int64)
+        for lo, hi in zip(edges[:-1], edges[1:]):
+            if hi > lo:
+                extra.append(int(rng.integers(lo, hi)))
+    return np.unique(np.array(list(fixed) + extra, dtype=np.int64))
+
+
+class Guarded:
+    """A CUDA tensor with 4 KiB of canary bytes before and after it: ``t`` is the tensor to
+    hand to the library, ``check()`` asserts that nothing was written outside it (stands in
+    for a memory checker on the output buffers)."""
+    PAD = 4096
+    CANARY = 0xA5
+
+    def __init__(self, shape, dtype):
+        import torch
+        self.torch = torch
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.n = n
+        self.raw = torch.full((self.PAD + ((n + 15) // 16) * 16 + self.PAD,), self.CANARY, dtype=torch.uint8,
+                              device="cuda")
+        self.t = self.raw[self.PAD:self.PAD + n].view(dtype).view(shape)
+
+    def check(self, label=""):
+        before = self.raw[:self.PAD]
+        after = self.raw[self.PAD + self.n:]
+        assert bool((before == self.CANARY).all()), f"{label}: bytes before the buffer were overwritten"
+        assert bool((after == self.CANARY).all()), f"{label}: bytes after the buffer were overwritten"

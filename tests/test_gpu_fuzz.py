@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import bf16_bits_to_f64, check_bf16_attention, check_fp8_attention
+from helpers import Guarded, bf16_bits_to_f64, check_bf16_attention, check_fp8_attention
 from paper_2609_13031_b200 import api
 from paper_2609_13031_b200 import workloads as W
 
@@ -46,8 +46,15 @@ def test_random_shapes_and_flags(i, cfg, n, m, fp8, half, gqa, test_only):
     x = {k: dev16(v) for k, v in g.items()}
     q_test = x["q_test"] if m else None
     f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    # every output buffer sits between canary bytes
+    guards = {"o_tr": Guarded((w.B, w.H, n, w.d), tdt), "o_te": Guarded((w.B, w.H, m, w.d), tdt)}
     if fp8:
-        o = api.quantize_qkv(x["q_train"], x["k"], x["v"], q_test, ws)
+        for name, rows in (("q8", n), ("k8", n), ("v8", n), ("t8", m)):
+            guards[name] = Guarded((w.B, w.H, rows, w.d), torch.uint8)
+        for name in ("sq", "sk", "sv"):
+            guards[name] = Guarded((w.B, w.H), torch.float32)
+        o = api.quantize_qkv(x["q_train"], x["k"], x["v"], q_test, ws,
+                             out={k: guards[k].t for k in ("q8", "k8", "v8", "t8", "sq", "sk", "sv")})
         q8, sq = oracle.quantize(g["q_train"], dtype16=dtype16)
         k8, sk = oracle.quantize(g["k"], dtype16=dtype16)
         v8, sv = oracle.quantize(g["v"], dtype16=dtype16)
@@ -58,10 +65,16 @@ def test_random_shapes_and_flags(i, cfg, n, m, fp8, half, gqa, test_only):
             t8, _ = oracle.quantize(g["q_test"], scale_in=sq, dtype16=dtype16)
             assert np.array_equal(o["t8"].cpu().numpy(), t8)
         o_tr, o_te = api.icl_forward_fp8(None if test_only else o["q8"], o["t8"] if m else None, o["k8"], o["v8"],
-                                         o["sq"], o["sk"], o["sv"], ws, flags=flags, out_dtype=tdt)
+                                         o["sq"], o["sk"], o["sv"], ws, flags=flags,
+                                         out_train=None if test_only else guards["o_tr"].t,
+                                         out_test=guards["o_te"].t if m else None)
     else:
-        o_tr, o_te = api.icl_forward_bf16(None if test_only else x["q_train"], q_test, x["k"], x["v"], ws, flags=flags)
+        o_tr, o_te = api.icl_forward_bf16(None if test_only else x["q_train"], q_test, x["k"], x["v"], ws, flags=flags,
+                                          out_train=None if test_only else guards["o_tr"].t,
+                                          out_test=guards["o_te"].t if m else None)
     assert api.last_device_status(ws) == (0, 0)
+    for name, gd in guards.items():
+        gd.check(f"fuzz{i} {name}")
     label = f"fuzz{i}/{cfg}/{n}+{m}/fp8={fp8}/half={half}/gqa={gqa}/test_only={test_only}"
     for name, out, nq in (("train", o_tr, n), ("test", o_te, m)):
         if nq == 0 or (name == "train" and test_only):

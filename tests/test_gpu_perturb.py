@@ -75,3 +75,42 @@ def test_coordinated_noise_feeds_both_attention_calls():
     o_tr, o_te = api.icl_forward_bf16(q_train, q_test, k, v, ws)
     assert api.last_device_status(ws) == (0, 0)
     assert torch.equal(o_te[:, :, 9], o_tr[:, :, 200])
+
+
+def test_gpu_noise_field_statistics():
+    """What Eq. 3 fixes, checked on the GPU output itself (not through the oracle, which
+    restates the same counter-based generator): rho is the head RMS, and the standardised
+    noise (out - x) / (eps * rho) has zero mean, unit variance, normal kurtosis, and is
+    uncorrelated across heads, across neighbouring elements and across streams; the
+    perturbation is linear in eps."""
+    B, H, R, d = 1, 4, 4096, 64
+    rng = np.random.default_rng(11)
+    # per-head constant magnitudes with random signs: rho is known exactly (the constant), and
+    # with eps = 8 the noise dominates the bf16 rounding of the sum
+    consts = np.array([0.5, 1.0, 2.0, 3.0])
+    xs = np.sign(rng.standard_normal((B, H, R, d))) * consts[None, :, None, None]
+    x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16).cuda()
+    ws = api.new_workspace(B, H)
+    eps = 8.0
+    out, rho = api.perturb(x, eps, seed=123, stream_id=0, workspace=ws)
+    out2, _ = api.perturb(x, eps, seed=123, stream_id=1, workspace=ws)
+    assert np.allclose(rho.cpu().numpy()[0], consts, rtol=1e-6)          # rho = sqrt(mean x^2) of the head
+    xf = x.double().cpu().numpy()
+    z = (out.double().cpu().numpy() - xf) / (eps * consts[None, :, None, None])
+    z2 = (out2.double().cpu().numpy() - xf) / (eps * consts[None, :, None, None])
+    n = R * d
+    for h in range(H):
+        zh = z[0, h].ravel()
+        assert abs(zh.mean()) < 5 / np.sqrt(n)
+        assert abs(zh.var() - 1.0) < 0.02                                # bf16 rounding of the sum adds < 1 %
+        assert abs(((zh - zh.mean()) ** 4).mean() / zh.var() ** 2 - 3.0) < 0.1
+        # neighbouring elements come from one Box-Muller pair: still uncorrelated
+        assert abs(np.corrcoef(zh[0::2], zh[1::2])[0, 1]) < 5 / np.sqrt(n / 2)
+        # the same positions of another head, and of another stream, are independent draws
+        assert abs(np.corrcoef(zh, z[0, (h + 1) % H].ravel())[0, 1]) < 5 / np.sqrt(n)
+        assert abs(np.corrcoef(zh, z2[0, h].ravel())[0, 1]) < 5 / np.sqrt(n)
+    # linear in eps: half the strength, half the displacement (up to the rounding of the result)
+    half, _ = api.perturb(x, eps / 2, seed=123, stream_id=0, workspace=ws)
+    zhalf = (half.double().cpu().numpy() - xf) / (eps / 2 * consts[None, :, None, None])
+    assert np.abs(zhalf - z).mean() < 0.02 and np.corrcoef(zhalf.ravel(), z.ravel())[0, 1] > 0.999
+    assert api.last_device_status(ws) == (0, 0)

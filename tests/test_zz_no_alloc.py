@@ -6,7 +6,8 @@ or a memory pool that already owns the GPU).  Its scratch is a fixed array insid
 the library that every call shares and that keeps the previous call's contents,
 so the check runs two different tensors back to back: stale maxima left by the
 first call would corrupt the scales of the second.  Results must equal the
-regular entry point's bit for bit, which is the bar all quantizer tests use.
+regular entry point's bit for bit, which is the bar all quantizer tests use, and
+they are compared with the CPU oracle directly as well.
 
 This file is named to be collected last; it also passes when run on its own.
 """
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_13031_b200 import api
 from paper_2609_13031_b200 import workloads as W
 
@@ -49,6 +51,12 @@ def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
     assert torch.equal(scale, ref_big_s) and torch.equal(out, ref_big)
     assert torch.equal(scale2, ref_small_s) and torch.equal(out2, ref_small)
     assert torch.equal(scale3, ref_big_s) and torch.equal(out3, ref_test)
+    # the oracle itself, not only the other GPU entry point
+    small_bits = small.view(torch.int16).cpu().numpy().view(np.uint16)
+    for got, got_s, bits, s_in in ((out, scale, g["k"], None), (out2, scale2, small_bits, None),
+                                   (out3, scale3, g["q_test"], scale.cpu().numpy())):
+        want, want_s = oracle.quantize(bits, scale_in=s_in)
+        assert np.array_equal(got.cpu().numpy(), want) and np.array_equal(got_s.cpu().numpy(), want_s)
     # and once more in the opposite order
     api.quantize_noalloc(small, out2, scale2)
     api.quantize_noalloc(big, out, scale)
