@@ -162,9 +162,11 @@ __device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64
     uint4* oh = out + (int64_t)blockIdx.y * pairs_per_head;
     int64_t stride = (int64_t)gridDim.x * kThreads;
     // A bf16 subnormal (below 2^-126) is no (1.m) * 2^e; it can only give a non-zero code
-    // (|x/s| >= 2^-10) if s < 2^-116.  Such a head, and one with a non-finite scale, takes the
-    // per-element division.
-    const bool direct = !(s >= 1e-30f && s <= 3e38f);
+    // (|x/s| >= 2^-10) if s < 2^-116.  And (1.m) / s must itself be a normal number for the
+    // table entry to be the exact quotient's mantissa: s < 2^126.  Heads outside a scale range
+    // kept well inside both limits (and given scales that are zero, negative or not finite)
+    // take the per-element division.
+    const bool direct = !(s >= 1e-30f && s <= 1e30f);
     // walk the head from its end towards its start
     for (int64_t r = (int64_t)blockIdx.x * kThreads + threadIdx.x; r < pairs_per_head; r += stride) {
         int64_t i = pairs_per_head - 1 - r;
@@ -368,7 +370,7 @@ __global__ void __launch_bounds__(kOneThreads) quantize_one_launch_kernel(const 
             for (int mnt = threadIdx.x; mnt < kTab; mnt += kOneThreads)
                 tab[mnt] = __fdiv_rn(__uint_as_float(0x3f800000u | ((uint32_t)mnt << (23 - T::kMantBits))), s);
             __syncthreads();
-            const bool direct = !(s >= 1e-30f && s <= 3e38f);
+            const bool direct = !(s >= 1e-30f && s <= 1e30f);
             const uint4* xh = a.b.x[z] + head * pph * 2;
             uint4* oh = a.b.out[z] + head * pph;
             auto convert = [&](const uint4& u, const uint4& v) {

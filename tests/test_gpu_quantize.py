@@ -173,3 +173,26 @@ def test_fused_qkv_query_scale_from_all_rows(extra):
     assert np.array_equal(o["q8"].cpu().numpy(), rq) and np.array_equal(o["t8"].cpu().numpy(), rt)
     rk, rsk = oracle.quantize(g["k"])
     assert np.array_equal(o["k8"].cpu().numpy(), rk) and np.array_equal(o["sk"].cpu().numpy(), rsk)
+
+
+@pytest.mark.parametrize("scale", [1e-38, 3e-31, 1e-30, 7.3e-12, 1.0, 6.5e11, 1e30, 3e30, 2.9e38])
+def test_given_scales_across_the_exponent_range(scale):
+    """A given scale anywhere in the fp32 range (the conversion takes its quotients from a
+    per-mantissa table inside a safe scale range and divides per element outside it): codes
+    equal the oracle's, for inputs that span the whole bf16 exponent range, subnormals, zeros
+    and both signs included."""
+    rng = np.random.default_rng(17)
+    bits = rng.integers(0, 0x7F80, size=(1, 2, 64, 64), dtype=np.uint16)       # every finite magnitude
+    bits[0, 0, 0, :8] = [0x0000, 0x0001, 0x007F, 0x0080, 0x7F7F, 0x3F80, 0x0040, 0x7F00]
+    bits |= (rng.integers(0, 2, size=bits.shape, dtype=np.uint16) << 15)
+    # values around the scale itself, where the codes are neither zero nor saturated
+    near = np.clip(rng.standard_normal((1, 2, 64, 64)) * scale * 100, -3e38, 3e38).astype(np.float32)
+    near_bits = f32_to_bf16_bits(near).reshape(1, 2, 64, 64)
+    x = np.concatenate([bits, near_bits], axis=2)
+    s_in = np.full((1, 2), scale, dtype=np.float32)
+    ws = api.new_workspace(1, 2)
+    codes, s_out = api.quantize(to_dev(x), ws, scale_in=torch.from_numpy(s_in).cuda())
+    want, _ = oracle.quantize(x, scale_in=s_in)
+    got = codes.cpu().numpy()
+    assert np.array_equal(got, want), np.argwhere(got != want)[:5]
+    assert np.array_equal(s_out.cpu().numpy(), s_in)
