@@ -93,7 +93,10 @@ def check_bf16_case(w, n_sample=None):
         rows = np.arange(nq) if n_sample is None else sample_rows(nq, n_sample, w.seed)
         A, Abs, _ = oracle.icl_attention_rows(q, g["k"], g["v"], rows)
         got = out_to_f64(out[:, :, torch.from_numpy(rows).cuda()])
-        check_bf16_attention(got, A, Abs, label=f"{w.name}/{name}")
+        st = check_bf16_attention(got, A, Abs, label=f"{w.name}/{name}")
+        print(f"parity bf16 {w.name}/{name}: rows/head {rows.size} max_abs {st['max_abs']:.4g} mean_abs {st['mean_abs']:.4g} "
+              f"max_norm {st['max_norm']:.4g} mean_norm {st['mean_norm']:.4g} rel_rms {st['rel_rms']:.4g} "
+              f"bound_ratio {st['bound_ratio']:.3f}")
 
 
 # ---- FP8 path ---------------------------------------------------------------------
