@@ -190,6 +190,17 @@ def oracle_sample(w, rows_per_head: int, seed: int = 0):
     return flops / seconds / 1e12, info
 
 
+# one step of either arm: the same work, named the same way
+STEP_LABEL = "quantize Q_train, K, V (per-head absmax) and Q_test (train-query scale), then ICL attention train->train + test->train"
+
+
+def l2_label(w) -> str:
+    """Timing hygiene: how the inputs of a step relate to the 126 MB L2 (no flush between steps
+    where they exceed it; smaller workloads say so)."""
+    mb = 2.0 * w.B * w.H * w.d * (3 * w.n_train + w.n_test) / 1e6
+    return "bf16 inputs %.0f MB, %s the 126 MB L2; no flush between steps" % (mb, "larger than" if mb > 126 else "smaller than")
+
+
 def workload_label(w) -> str:
     return f"{w.name}: B={w.B} H={w.H} d={w.d} n_train={w.n_train} n_test={w.n_test}"
 
@@ -211,9 +222,9 @@ def run_reference(args, w):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * sec, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_label(w),
-                   "step": "oracle quantize + exact attention over the dequantized operands, "
-                           "a bounded sample of the step's rows"},
+        "config": {"workload": workload_label(w), "step": STEP_LABEL, "l2": l2_label(w)},
+        "impl_detail": "oracle quantize + exact attention over the dequantized operands, a bounded sample of "
+                       "the step's query rows per timed step",
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": info["cores"], "kind": "oracle",
                          "sample": info["sample"]},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -515,11 +526,10 @@ def main():
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
             "data": "synthetic",
-            "config": {"workload": workload_label(w),
-                       "step": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
-                       "l2": "inputs larger than L2 (bf16 inputs %.0f MB)" % (h2d / 1e6),
-                       "preroll": "%d untimed steps (%.1f s) under the same load before the timed steps" % (pre_n, pre_s),
-                       "replicas": world},
+            "config": {"workload": workload_label(w), "step": STEP_LABEL, "l2": l2_label(w)},
+            "impl_detail": {"calls": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
+                            "preroll": "%d untimed steps (%.1f s) under the same load before the timed steps" % (pre_n, pre_s),
+                            "replicas": world},
             "clocks": clocks,
             "e2e": {"value": world * tf(ms_e2e), "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,

@@ -162,7 +162,7 @@ def test_bf16_c2_sampled():
 
 
 def test_bf16_c3_full_size_sampled():
-    check_bf16_case(W.CONFIGS["C3"], n_sample=24)
+    check_bf16_case(W.CONFIGS["C3"], n_sample=128)
 
 
 # ---- structure of the ICL layer -------------------------------------------------------
