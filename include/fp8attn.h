@@ -201,6 +201,10 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
  * rows take the split path depends on the sizes of the call, so a row's result
  * is no longer bit-identical across calls with different n_test.
  *
+ * Calls with this flag belong on one stream: run from two streams at the same time they
+ * stalled a B200 (the main grid is released early behind the split grid and waits for it
+ * before it exits; the cause of the stall was not established).
+ *
  * Unknown flag bits return FP8ATTN_ERR_INVALID_ARG.  flags = 0 is the plain call.
  */
 #define FP8ATTN_TEST_ROWS_USE_KV_HEAD0 1u
@@ -282,6 +286,54 @@ int fp8attn_perturb(const void* x_bf16, int B, int H, int64_t rows, int d,
 int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int d,
                              const float* scale_in, void* x_fp8, float* scale_out,
                              void* cuda_stream);
+
+/* One whole step of the path from HOST memory to HOST memory: the four tensors of an
+ * ICL attention call are copied to the device, quantized (fp8attn_quantize_qkv, paper
+ * Eq. 2 with the shared train-query scale), both attention calls run
+ * (fp8attn_icl_forward_ex with FP8ATTN_SPLIT_TAIL), and the 16-bit results are copied
+ * back.  The paper has no counterpart; this is the form a caller with host-resident
+ * tables uses, and the one the end-to-end latency of a call is measured on.
+ *
+ * Heads are independent in every step of the path, so a large call is cut into up to 8
+ * chunks of whole heads that run as a pipeline on three internal streams (copy-in of the
+ * next chunk, compute of the current one, copy-out of the previous one overlap; two sets
+ * of device buffers alternate).  Calls whose 16-bit inputs total less than 32 MB, and
+ * calls with FP8ATTN_HOST_ONE_CHUNK, run as one chunk.  Results are those of the
+ * device-pointer calls on the same data (a chunk is a call with B = 1 and the chunk's
+ * heads; with FP8ATTN_SPLIT_TAIL, which rows take the split path depends on the chunking).
+ *
+ *   q_train, k, v  in  HOST bf16 [B,H,n_train,d]    q_test in HOST bf16 [B,H,n_test,d] (NULL iff n_test == 0)
+ *   out_train      out HOST bf16 [B,H,n_train,d]    out_test out HOST bf16 [B,H,n_test,d] (NULL iff n_test == 0)
+ *   device_scratch DEVICE memory owned by the caller, 256-byte aligned, at least
+ *                  fp8attn_host_step_scratch_bytes(...) bytes with the same sizes and flags;
+ *                  its contents on entry do not matter
+ *   flags          FP8ATTN_HOST_ONE_CHUNK (no pipeline), FP8ATTN_HOST_FP16 (all 16-bit tensors
+ *                  are IEEE fp16); other bits: FP8ATTN_ERR_INVALID_ARG
+ *
+ * The host buffers should be page-locked: copies from pageable memory are staged by the
+ * CUDA runtime and do not overlap.  The call only enqueues work (after everything already
+ * in `cuda_stream`; `cuda_stream` continues after the last copy-out), so the host buffers
+ * must stay valid, and the outputs are complete, once `cuda_stream` has been synchronised.
+ * Host steps are ordered on the GPU in the order in which they were called, also when they
+ * were given different streams: one pipelined call keeps the copy engines and the SMs busy,
+ * and two of them side by side (attention launches with FP8ATTN_SPLIT_TAIL from two streams
+ * at once) stalled the GPU when it was tried, so the library does not let it happen.
+ * The library allocates no device memory here either; it creates and releases three
+ * streams and a few events per call.  fp8attn_host_step_status synchronises `cuda_stream`
+ * and returns the device status of the call's workspaces (inside the scratch), like
+ * fp8attn_last_device_status.  fp8attn_host_step_chunks returns the number of chunks
+ * the call is cut into (0 for unsupported sizes, like the scratch size). */
+#define FP8ATTN_HOST_ONE_CHUNK 1u
+#define FP8ATTN_HOST_FP16 2u
+size_t fp8attn_host_step_scratch_bytes(int B, int H, int64_t n_train, int64_t n_test, int d,
+                                       uint32_t flags);
+int fp8attn_host_step_chunks(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags);
+int fp8attn_icl_step_host(const void* q_train, const void* k, const void* v, const void* q_test,
+                          int B, int H, int64_t n_train, int64_t n_test, int d,
+                          float softmax_scale, uint32_t flags, void* out_train, void* out_test,
+                          void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
+int fp8attn_host_step_status(void* device_scratch, int B, int H, int64_t n_train, int64_t n_test,
+                             int d, uint32_t flags, void* cuda_stream, uint32_t* detail);
 
 /* Bytes of workspace the calls above need: a few KB for the status words and the
  * per-head accumulators (all that is returned for n_train = 0), plus, for

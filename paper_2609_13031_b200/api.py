@@ -25,6 +25,8 @@ EXPORTS = (
     "fp8attn_icl_forward_ex", "bf16attn_icl_forward_ex", "fp8attn_gate_use_fp8",
     "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex", "fp8attn_perturb",
     "fp8attn_selftest_wait_timeout", "fp8attn_quantize_ex",
+    "fp8attn_icl_step_host", "fp8attn_host_step_scratch_bytes", "fp8attn_host_step_chunks",
+    "fp8attn_host_step_status",
 )
 # flags of fp8attn_quantize_ex / fp8attn_quantize_qkv_ex
 QUERY_SCALE_FROM_ALL_ROWS = 1
@@ -37,6 +39,9 @@ TEST_ROWS_ONLY = 2
 IO_FP16 = 4
 SPLIT_TAIL = 8
 GATE_TRAIN_ROWS = 8192
+# flags of fp8attn_icl_step_host
+HOST_ONE_CHUNK = 1
+HOST_FP16 = 2
 
 _lib = None
 
@@ -99,6 +104,14 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_status_string.argtypes = [i32]
     lib.fp8attn_launch_count.restype = ctypes.c_uint64
     lib.fp8attn_launch_count.argtypes = []
+    lib.fp8attn_host_step_scratch_bytes.restype = sz
+    lib.fp8attn_host_step_scratch_bytes.argtypes = [i32, i32, i64, i64, i32, u32]
+    lib.fp8attn_host_step_chunks.restype = i32
+    lib.fp8attn_host_step_chunks.argtypes = [i32, i32, i64, i64, i32, u32]
+    lib.fp8attn_icl_step_host.restype = i32
+    lib.fp8attn_icl_step_host.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, f32, u32, vp, vp, vp, sz, vp]
+    lib.fp8attn_host_step_status.restype = i32
+    lib.fp8attn_host_step_status.argtypes = [vp, i32, i32, i64, i64, i32, u32, vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = lib
     return lib
 
@@ -324,6 +337,60 @@ def last_device_status(workspace: torch.Tensor):
     """Synchronise the current stream; returns (status, detail) recorded by the kernels."""
     detail = ctypes.c_uint32(0)
     rc = load().fp8attn_last_device_status(_ptr(workspace), _stream(), ctypes.byref(detail))
+    return int(rc), int(detail.value)
+
+
+def _host_dims(q_train, k, v, q_test):
+    assert k.dim() == 4 and not k.is_cuda and k.is_contiguous() and _is16(k), "expected contiguous host [B,H,rows,d]"
+    for t in (q_train, v):
+        assert t.shape == k.shape and t.dtype == k.dtype and not t.is_cuda and t.is_contiguous()
+    B, H, n_train, d = k.shape
+    n_test = 0
+    if q_test is not None:
+        assert q_test.dtype == k.dtype and not q_test.is_cuda and q_test.is_contiguous()
+        assert q_test.shape[:2] == k.shape[:2] and q_test.shape[3] == d
+        n_test = q_test.shape[2]
+    return B, H, n_train, n_test, d
+
+
+def host_step_scratch_bytes(B: int, H: int, n_train: int, n_test: int, d: int, flags: int = 0) -> int:
+    return int(load().fp8attn_host_step_scratch_bytes(B, H, n_train, n_test, d, int(flags)))
+
+
+def host_step_chunks(B: int, H: int, n_train: int, n_test: int, d: int, flags: int = 0) -> int:
+    return int(load().fp8attn_host_step_chunks(B, H, n_train, n_test, d, int(flags)))
+
+
+def icl_step_host(q_train, k, v, q_test, scratch: torch.Tensor, softmax_scale: float = 0.0, flags: int = 0,
+                  out_train=None, out_test=None):
+    """fp8attn_icl_step_host: quantize + both attention calls from HOST tensors (page-locked
+    for overlap) to HOST results, pipelined over chunks of heads.  ``scratch``: uint8 CUDA
+    tensor of at least ``host_step_scratch_bytes`` bytes.  Enqueues on the current stream and
+    returns (out_train, out_test) host tensors that are complete once that stream has been
+    synchronised."""
+    B, H, n_train, n_test, d = _host_dims(q_train, k, v, q_test)
+    if k.dtype == torch.float16:
+        flags |= HOST_FP16
+    if out_train is None:
+        out_train = torch.empty(k.shape, dtype=k.dtype).pin_memory()
+    if out_test is None and n_test > 0:
+        out_test = torch.empty(q_test.shape, dtype=k.dtype).pin_memory()
+    for t in (out_train, out_test):
+        assert t is None or (not t.is_cuda and t.is_contiguous() and t.dtype == k.dtype)
+    assert scratch.is_cuda and scratch.dtype == torch.uint8
+    rc = load().fp8attn_icl_step_host(_ptr(q_train), _ptr(k), _ptr(v), _ptr(q_test) if n_test else None,
+                                      B, H, n_train, n_test, d, float(softmax_scale), int(flags),
+                                      _ptr(out_train), _ptr(out_test) if n_test else None,
+                                      _ptr(scratch), scratch.numel(), _stream())
+    _check("fp8attn_icl_step_host", rc)
+    return out_train, out_test
+
+
+def host_step_status(scratch: torch.Tensor, B: int, H: int, n_train: int, n_test: int, d: int, flags: int = 0):
+    """Synchronise the current stream; (status, detail) of the workspaces of a host step."""
+    detail = ctypes.c_uint32(0)
+    rc = load().fp8attn_host_step_status(_ptr(scratch), B, H, n_train, n_test, d, int(flags), _stream(),
+                                         ctypes.byref(detail))
     return int(rc), int(detail.value)
 
 

@@ -40,6 +40,24 @@ def test_host_only_entry_points():
     assert api.workspace_bytes(0, 4) == 0
 
 
+def test_host_step_plan_is_host_only_arithmetic():
+    """Chunking of the host-to-host step: whole heads, at most 8 chunks, one chunk for small
+    calls or on request; two buffer sets when pipelined, so the scratch shrinks with chunking."""
+    api.load()
+    c3 = (1, 8, 65536, 16384, 128)
+    assert api.host_step_chunks(*c3) == 8 and api.host_step_chunks(*c3, api.HOST_ONE_CHUNK) == 1
+    assert api.host_step_chunks(1, 2, 512, 128, 64) == 1                  # small: nothing to overlap
+    assert api.host_step_chunks(4, 4, 262144, 65536, 64) == 8             # 16 heads, two per chunk
+    assert api.host_step_chunks(1, 11, 8192, 1100, 128) == 6              # ragged last chunk
+    assert api.host_step_chunks(1, 1, 1 << 20, 0, 64) == 1                # one head cannot be cut
+    one = api.host_step_scratch_bytes(*c3, api.HOST_ONE_CHUNK)
+    piped = api.host_step_scratch_bytes(*c3)
+    per_head = (3 * 65536 + 16384) * 128 * (2 + 1) + (65536 + 16384) * 128 * 2   # inputs, codes, outputs
+    assert one >= 8 * per_head and 2 * per_head <= piped < one / 2
+    assert one % 256 == 0 and piped % 256 == 0
+    assert api.host_step_scratch_bytes(1, 8, 0, 16, 64) == 0 and api.host_step_scratch_bytes(1, 8, 64, 16, 96) == 0
+
+
 def test_dispatch_gate_matches_the_paper_constant():
     import os
     from helpers import read_golden_table
