@@ -404,85 +404,76 @@ def main():
         ms_bf16 = max_over_ranks(float(np.mean(t_bf16)))
     sampler.stop()
 
-    # ---- end to end: pinned host inputs -> device -> path -> host outputs, every step ----
-    # Every step copies its own inputs from pinned host memory and its own results back.  The
-    # copies of neighbouring steps overlap the compute of the current one: three streams
-    # (copy-in, compute, copy-out) and two sets of device buffers, ordered by events.
-    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    sets = []
-    for _ in range(2):
-        d_in = {k: torch.empty_like(v, device="cuda") for k, v in host.items()}
-        d_buf = {k: torch.empty_like(v) for k, v in buf.items()}
-        sets.append((d_in, d_buf))
-    free_in = [None, None]      # event: compute no longer reads this input set
-    free_out = [None, None]     # event: copy-out no longer reads this output set
+    # ---- end to end: the host-to-host call of the C-ABI (fp8attn_icl_step_host) ----
+    # Every step hands pinned HOST tensors to the library and gets HOST results back; the call
+    # copies in, quantizes, runs both attention calls and copies out, pipelined over chunks of
+    # heads.  Throughput: steps alternate between two streams (own device scratch and own host
+    # result buffers each), so that the copies of one step overlap the kernels of the other.
+    shape = (w.B, w.H, w.n_train, w.n_test, w.d)
+    n_slots = 2
+    slots = []
+    for _ in range(n_slots):
+        slots.append({"stream": torch.cuda.Stream(),
+                      "scratch": torch.empty(api.host_step_scratch_bytes(*shape), dtype=torch.uint8, device="cuda"),
+                      "o_tr": torch.empty_like(host_out["o_tr"]).pin_memory(),
+                      "o_te": torch.empty_like(host_out["o_te"]).pin_memory()})
+
+    def host_step(slot, flags=0, scratch=None):
+        api.icl_step_host(host["q_train"], host["k"], host["v"], host["q_test"],
+                          slot["scratch"] if scratch is None else scratch, flags=flags,
+                          out_train=slot["o_tr"], out_test=slot["o_te"])
 
     def e2e_run(n):
         for i in range(n):
-            d_in, d_buf = sets[i % 2]
-            with torch.cuda.stream(s_in):
-                if free_in[i % 2] is not None:
-                    s_in.wait_event(free_in[i % 2])
-                for k in host:
-                    d_in[k].copy_(host[k], non_blocking=True)
-                e_in = torch.cuda.Event()
-                e_in.record(s_in)
-            with torch.cuda.stream(s_cmp):
-                s_cmp.wait_event(e_in)
-                if free_out[i % 2] is not None:
-                    s_cmp.wait_event(free_out[i % 2])
-                api.quantize_qkv(d_in["q_train"], d_in["k"], d_in["v"], d_in["q_test"], ws, out=d_buf)
-                api.icl_forward_fp8(d_buf["q8"], d_buf["t8"], d_buf["k8"], d_buf["v8"], d_buf["sq"],
-                                    d_buf["sk"], d_buf["sv"], ws, 0.0, out_train=d_buf["o_tr"],
-                                    out_test=d_buf["o_te"], flags=fwd_flags)
-                e_c = torch.cuda.Event()
-                e_c.record(s_cmp)
-                free_in[i % 2] = e_c
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(e_c)
-                host_out["o_tr"].copy_(d_buf["o_tr"], non_blocking=True)
-                host_out["o_te"].copy_(d_buf["o_te"], non_blocking=True)
-                e_o = torch.cuda.Event()
-                e_o.record(s_out)
-                free_out[i % 2] = e_o
+            slot = slots[i % n_slots]
+            with torch.cuda.stream(slot["stream"]):
+                host_step(slot)
 
     def join_streams():
         cur = torch.cuda.current_stream()
-        for st in (s_in, s_cmp, s_out):
-            cur.wait_stream(st)
+        for slot in slots:
+            cur.wait_stream(slot["stream"])
 
-    for st in (s_in, s_cmp, s_out):
-        st.wait_stream(torch.cuda.current_stream())
+    sync_all()
+    for slot in slots:
+        slot["stream"].wait_stream(torch.cuda.current_stream())
     e2e_run(2)
     join_streams()
     sync_all()
     n_e2e = max(4, min(args.steps, 20))
     a, b = ev(), ev()
     a.record()
-    for st in (s_in, s_cmp, s_out):
-        st.wait_stream(torch.cuda.current_stream())
+    for slot in slots:
+        slot["stream"].wait_stream(torch.cuda.current_stream())
     e2e_run(n_e2e)
     join_streams()
     b.record()
     sync_all()
     ms_e2e = max_over_ranks(a.elapsed_time(b)) / n_e2e
+    for slot in slots:
+        st = api.host_step_status(slot["scratch"], *shape)
+        if st != (0, 0):
+            raise RuntimeError(f"device status after the end-to-end steps: {st}")
     h2d = sum(t.numel() * t.element_size() for t in host.values())
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+    # ---- one call, host to host, wall clock: the pipelined call, and the same call as one chunk ----
+    def single_call(flags, scratch):
+        ts = []
+        for i in range(max(4, min(args.steps, 6))):
+            sync_all()
+            t0 = time.perf_counter()
+            host_step(slots[0], flags=flags, scratch=scratch)
+            torch.cuda.synchronize()
+            if i > 0:                       # the first call of a kind pays its set-up
+                ts.append(1e3 * (time.perf_counter() - t0))
+        return max_over_ranks(float(np.median(ts)))
 
-    # ---- one call, host to host, nothing overlapped: copy in, quantize, attention, copy out ----
-    single = []
-    for _ in range(max(3, min(args.steps, 5))):
-        sync_all()
-        t0 = time.perf_counter()
-        for k in host:
-            dev[k].copy_(host[k], non_blocking=True)
-        quantize_all()
-        attention_fp8()
-        host_out["o_tr"].copy_(buf["o_tr"], non_blocking=True)
-        host_out["o_te"].copy_(buf["o_te"], non_blocking=True)
-        torch.cuda.synchronize()
-        single.append(1e3 * (time.perf_counter() - t0))
-    ms_single = max_over_ranks(float(np.median(single)))
+    ms_single = single_call(0, slots[0]["scratch"])
+    slots[1]["scratch"] = None              # make room for the unpipelined call's larger scratch
+    one_chunk = torch.empty(api.host_step_scratch_bytes(*shape, api.HOST_ONE_CHUNK), dtype=torch.uint8, device="cuda")
+    ms_single_one_chunk = single_call(api.HOST_ONE_CHUNK, one_chunk)
+    n_chunks = api.host_step_chunks(*shape)
+    del one_chunk
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----
     cpu_baseline = None
@@ -533,9 +524,13 @@ def main():
             "clocks": clocks,
             "e2e": {"value": world * tf(ms_e2e), "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
-                    "kind": "pipelined throughput: copies of neighbouring steps overlap the compute (3 streams, 2 buffer sets)",
+                    "kind": "fp8attn_icl_step_host on pinned host tensors, steps alternating between two streams "
+                            "(copies of one step overlap the kernels of the other)",
+                    "chunks_per_call": n_chunks,
                     "single_call_ms": ms_single, "single_call_value": world * tf(ms_single),
-                    "single_call_kind": "median host-to-host latency of one step, nothing overlapped"},
+                    "single_call_kind": "median wall-clock latency of one fp8attn_icl_step_host call, host to host, "
+                                        "synchronised before and after",
+                    "single_call_one_chunk_ms": ms_single_one_chunk},
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "kernel": "icl_attention_kernel<fp8>",
                          "achieved": tf_attn, "peak": peak_fp8, "unit": "TFLOP/s",

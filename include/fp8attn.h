@@ -314,10 +314,11 @@ int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int
  * CUDA runtime and do not overlap.  The call only enqueues work (after everything already
  * in `cuda_stream`; `cuda_stream` continues after the last copy-out), so the host buffers
  * must stay valid, and the outputs are complete, once `cuda_stream` has been synchronised.
- * Host steps are ordered on the GPU in the order in which they were called, also when they
- * were given different streams: one pipelined call keeps the copy engines and the SMs busy,
- * and two of them side by side (attention launches with FP8ATTN_SPLIT_TAIL from two streams
- * at once) stalled the GPU when it was tried, so the library does not let it happen.
+ * Calls made on different streams (each with its own scratch and host buffers) may be in
+ * flight together: their copies overlap the other call's kernels.  Their kernels do not
+ * overlap: the library orders the kernels of host steps on a device in the order of the
+ * calls (attention launches with FP8ATTN_SPLIT_TAIL from two streams at once stalled the
+ * GPU when it was tried).
  * The library allocates no device memory here either; it creates and releases three
  * streams and a few events per call.  fp8attn_host_step_status synchronises `cuda_stream`
  * and returns the device status of the call's workspaces (inside the scratch), like

@@ -18,13 +18,14 @@ constexpr int64_t kPipelineMinBytes = 32ll << 20;   // 16-bit input bytes below 
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-// Host steps never overlap on a GPU: every call waits for the end of the one before it on the
-// same device, whatever stream that was made on.  (Two pipelined calls running their attention
-// launches side by side from different streams stalled the GPU when it was tried; one call
-// already keeps the copy engines and the SMs busy, so nothing is lost by ordering them.)
+// The kernels of two host steps never overlap on a GPU: the compute stream of every call waits
+// for the last kernel of the call before it on the same device, whatever stream that was made
+// on.  (Two pipelined calls running their attention launches side by side from different streams
+// stalled the GPU when it was tried.)  The copies of a call made on another stream are free to
+// overlap those kernels, which is all that two calls in flight can gain.
 constexpr int kMaxDevices = 64;
 std::mutex g_order_mutex;
-cudaEvent_t g_last_end[kMaxDevices] = {};
+cudaEvent_t g_last_compute[kMaxDevices] = {};
 
 struct Plan {
     int heads;            // B*H
@@ -147,13 +148,13 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
     // one call at a time enqueues, so that the order of the calls on the GPU is the order of the calls
     std::lock_guard<std::mutex> lock(g_order_mutex);
     if (rc == FP8ATTN_OK) {
-        // after the host step before this one on the device ...
-        if (g_last_end[dev] != nullptr) cu(cudaStreamWaitEvent(user, g_last_end[dev], 0));
-        // ... and after what the caller's stream holds so far
+        // everything of this call comes after what the caller's stream holds so far ...
         record(e_start, user);
         wait(s_in, e_start);
         wait(s_cmp, e_start);
         wait(s_out, e_start);
+        // ... and its kernels after those of the host step before it on the device
+        if (g_last_compute[dev] != nullptr) cu(cudaStreamWaitEvent(s_cmp, g_last_compute[dev], 0));
         char* base = static_cast<char*>(device_scratch);
         // the small head of each set's workspace (status words, counters, accumulators) starts at zero
         const size_t ws_head = fp8attn_workspace_bytes(1, p.chunk_heads, 0, 0, d);
@@ -202,19 +203,19 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
                                    cudaMemcpyDeviceToHost, s_out));
             record(e_o[c], s_out);
         }
+        // the last kernel of this call, for the next call's kernels to wait on
+        cudaEvent_t done = nullptr;
+        if (cu(cudaEventCreateWithFlags(&done, cudaEventDisableTiming)) && cu(cudaEventRecord(done, s_cmp))) {
+            if (g_last_compute[dev] != nullptr) cudaEventDestroy(g_last_compute[dev]);
+            g_last_compute[dev] = done;
+        } else if (done != nullptr) {
+            cudaEventDestroy(done);
+        }
         // the caller's stream continues after all three
         cudaStream_t all[3] = {s_in, s_cmp, s_out};
         for (int i = 0; i < 3; ++i) {
             record(e_end[i], all[i]);
             wait(user, e_end[i]);
-        }
-        // the end of this call, for the next one to wait on
-        cudaEvent_t done = nullptr;
-        if (cu(cudaEventCreateWithFlags(&done, cudaEventDisableTiming)) && cu(cudaEventRecord(done, user))) {
-            if (g_last_end[dev] != nullptr) cudaEventDestroy(g_last_end[dev]);
-            g_last_end[dev] = done;
-        } else if (done != nullptr) {
-            cudaEventDestroy(done);
         }
     }
     for (int c = 0; c < kMaxChunks; ++c) {

@@ -120,26 +120,28 @@ def test_fp16_tensors():
     check_against_oracle(w, g, o_tr, o_te, n_sample=32, dtype16="fp16")
 
 
-def test_calls_from_two_streams_are_ordered_by_the_library():
-    # host steps never overlap on the GPU: a call waits for the one before it, whatever its stream
+def test_calls_in_flight_on_two_streams():
+    # two calls, two streams, own scratch each: copies may overlap the other call's kernels; the
+    # library keeps the kernels of the two calls apart
     w = dataclasses.replace(W.CONFIGS["C3"].scaled(8192, 1024), B=1, H=6)
     ga, gb = W.generate(w), W.generate(dataclasses.replace(w, seed=w.seed + 100))
     xa = {k: host16(v) for k, v in ga.items()}
     xb = {k: host16(v) for k, v in gb.items()}
     nbytes = api.host_step_scratch_bytes(*shape_of(w))
-    # ONE scratch for both streams: only the library's ordering keeps the second call off it
-    scratch = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    sa, sb = torch.empty(nbytes, dtype=torch.uint8, device="cuda"), torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     st_a, st_b = torch.cuda.Stream(), torch.cuda.Stream()
-    with torch.cuda.stream(st_a):
-        a_tr, a_te = api.icl_step_host(xa["q_train"], xa["k"], xa["v"], xa["q_test"], scratch)
-    with torch.cuda.stream(st_b):
-        b_tr, b_te = api.icl_step_host(xb["q_train"], xb["k"], xb["v"], xb["q_test"], scratch)
-        st_b.synchronize()     # the second call's end implies the first one's
-    assert st_a.query()
-    assert api.host_step_status(scratch, *shape_of(w)) == (0, 0)
-    for x, tr, te in ((xa, a_tr, a_te), (xb, b_tr, b_te)):
-        ref_tr, ref_te = device_reference(w, x, 1)
-        assert torch.equal(tr, ref_tr) and torch.equal(te, ref_te)
+    res = []
+    for rep in range(2):        # the second pair is enqueued while the first is still running
+        with torch.cuda.stream(st_a):
+            res.append((xa, api.icl_step_host(xa["q_train"], xa["k"], xa["v"], xa["q_test"], sa)))
+        with torch.cuda.stream(st_b):
+            res.append((xb, api.icl_step_host(xb["q_train"], xb["k"], xb["v"], xb["q_test"], sb)))
+    torch.cuda.synchronize()
+    for scratch in (sa, sb):
+        assert api.host_step_status(scratch, *shape_of(w)) == (0, 0)
+    refs = {id(xa): device_reference(w, xa, 1), id(xb): device_reference(w, xb, 1)}
+    for x, (tr, te) in res:
+        assert torch.equal(tr, refs[id(x)][0]) and torch.equal(te, refs[id(x)][1])
 
 
 def test_argument_errors():
