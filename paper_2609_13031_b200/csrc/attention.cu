@@ -741,13 +741,15 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
     }
     // ---- teardown ----
-    // Launched behind the split grid with programmatic stream serialization, this grid
-    // completes only after that one has (and its writes are visible): the combine kernel,
-    // ordered behind this grid, may then read the split grid's partial results.
-    if (!kSplit) asm volatile("griddepcontrol.wait;" ::: "memory");
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    // Launched behind the split grid with programmatic stream serialization, this grid
+    // completes only after that one has (and its writes are visible): the combine kernel,
+    // ordered behind this grid, may then read the split grid's partial results.  The wait
+    // comes after the tensor memory has been given back: at d = 64 two CTAs fit on an SM, and
+    // a split CTA that shares the SM may be waiting for exactly that allocation.
+    if (!kSplit) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Combines the partial results of the split query blocks: with M = max_s c*m_s,
