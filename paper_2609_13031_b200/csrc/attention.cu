@@ -747,8 +747,10 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     // Launched behind the split grid with programmatic stream serialization, this grid
     // completes only after that one has (and its writes are visible): the combine kernel,
     // ordered behind this grid, may then read the split grid's partial results.  The wait
-    // comes after the tensor memory has been given back: at d = 64 two CTAs fit on an SM, and
-    // a split CTA that shares the SM may be waiting for exactly that allocation.
+    // comes after the tensor memory has been given back, so that a CTA never waits for another
+    // grid while it holds an allocation that a CTA of that grid could be blocked on.  (With
+    // 168 registers x 384 threads one CTA fills an SM's register file, so two CTAs do not
+    // share an SM today; the order keeps that from becoming a requirement.)
     if (!kSplit) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
