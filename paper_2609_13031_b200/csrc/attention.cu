@@ -17,8 +17,9 @@
 // probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 / fp16 in
 // the 16-bit path) to its own tensor-memory region, from where it is the A operand
 // of O_t += P_t V.  Where 512 columns cannot hold a separate P (bf16, d = 128),
-// P is written over S and Q K^T waits for P V instead.  The FP8 d = 128 path
-// steps over 96 keys at a time to make room for P.
+// P is written over S and Q K^T waits for P V instead.  In the FP8 d = 128 path the
+// two tiles take turns in one S region (S | P0 P0' | P1 P1' | O0 | O1), which leaves
+// room for 128-key steps and two P buffers per tile.
 //
 // Scale placement (FP8 path): x = (alpha * s_q * s_k * log2 e) * S feeds exp2;
 // the V scale and 1/rowsum are applied to O in the epilogue.
@@ -67,7 +68,14 @@ struct Cfg {
     static constexpr int kBoxes = kRowBytes / kBoxBytes;        // TMA boxes per tile
     static constexpr int kBoxCols = kBoxBytes / kES;
     static constexpr bool kSepP = !(kD == 128 && !kFp8);        // P in its own TMEM region
-    static constexpr int kKeys = (kFp8 && kD == 128) ? 96 : 128;  // keys per step
+    static constexpr int kKeys = 128;                           // keys per step
+    // FP8, d = 128: tensor memory has no room for two 128-column S tiles next to O and P, so
+    // the two query tiles take turns in ONE S region: a tile's scores sit there only from its
+    // Q K^T until its softmax warps have loaded them into registers (a small part of a step),
+    // and the tiles run about half a step apart anyway.  The Q K^T of one tile waits for the
+    // other tile's load instead of for its own.  (96-key steps with two S regions, the layout
+    // before this one, cost 3.6 % more time; 128-key steps with P written over S 6 % more.)
+    static constexpr bool kSharedS = kFp8 && kD == 128;
     static constexpr int kQTileBytes = kTileM * kRowBytes;
     static constexpr int kKVTileBytes = kKeys * kRowBytes;
     static constexpr int kUmmaK = 32 / kES;                     // elements per MMA K step
@@ -77,19 +85,20 @@ struct Cfg {
     static constexpr uint32_t kIdescQK = idesc(kFmt, kFmt, false, false, kTileM, kKeys);
     static constexpr uint32_t kIdescPV = idesc(kFmt, kFmt, false, true, kTileM, kD);
     static constexpr int kPCols = kKeys * kES / 4;              // TMEM columns of a P tile
-    // TMEM columns: S_t, then O_t at 256 + t*kD, P_t wherever 32-column-aligned room is left
-    static constexpr uint32_t kColS0 = 0, kColS1 = kKeys, kColO = 256;
-    static constexpr uint32_t kColP0 = !kSepP ? kColS0 : (kD == 128 ? 192u : 384u);
-    static constexpr uint32_t kColP1 = !kSepP ? kColS1 : (kD == 128 ? 224u : 384u + 64u);
+    // TMEM columns: S_t (one region for both tiles where shared), then O_t at 256 + t*kD, P_t
+    // wherever 32-column-aligned room is left
+    static constexpr uint32_t kColS0 = 0, kColS1 = kSharedS ? 0 : kKeys, kColO = 256;
+    static constexpr uint32_t kColP0 = !kSepP ? kColS0 : (kD == 128 ? 128u : 384u);
+    static constexpr uint32_t kColP1 = !kSepP ? kColS1 : (kD == 128 ? 192u : 384u + 64u);
     // Where tensor memory has room, P alternates between two buffers per tile (the second
     // kPCols columns after the first), so that writing P of one step never waits for the
     // P V of the step before.
-    static constexpr int kPBufs = (kFp8 && kD == 64) ? 2 : 1;
+    static constexpr int kPBufs = kFp8 ? 2 : 1;
     static constexpr bool kLateRescale = kD == 128;             // O rescale at the end of the step
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
     static constexpr int kPolyPer16 = kFp8 ? 4 : (kD == 128 ? 8 : 2);
-    static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= (kD == 128 ? 32 : 64)), "TMEM layout");
-    static_assert(!kSepP || kD == 64 || (2 * kKeys <= 192 && kPCols <= 32), "TMEM layout");
+    static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= 64), "TMEM layout");
+    static_assert(!kSepP || kD == 64 || (kSharedS && kKeys <= 128 && kPCols <= 32), "TMEM layout");
     static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
     static constexpr size_t kSmemBytes = (size_t)2 * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
 };
@@ -97,7 +106,7 @@ struct Cfg {
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], p_free[2], o_full[2];
+    uint64_t s_full[2], p_free[2], o_full[2], s_free[2];
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -377,6 +386,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             mbar_init(smem_u32(&bars.s_full[t]), 1);
             mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
+            mbar_init(smem_u32(&bars.s_free[t]), 4);   // one arrival per softmax warp of the tile
         }
         fence_mbar_init();
     }
@@ -464,7 +474,14 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         w.wait(smem_u32(&bars.q_full), 0, kWaitQFull);
         w.wait(smem_u32(&bars.k_full[0]), 0, kWaitKFull);
         tc_fence_after_sync();
-        for (int t = 0; t < ntiles; ++t) issue_qk(t, 0);
+        for (int t = 0; t < ntiles; ++t) {
+            if (C::kSharedS && t == 1) {
+                // the shared S region is tile 0's until its rows sit in registers
+                w.wait(smem_u32(&bars.s_free[0]), 0, kWaitSFree);
+                tc_fence_after_sync();
+            }
+            issue_qk(t, 0);
+        }
         if (elect_one()) mma_commit(smem_u32(&bars.k_empty[0]));
         __syncwarp();
         for (int j = 0; j + 1 < nkv; ++j) {
@@ -472,9 +489,20 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
             for (int t = 0; t < ntiles; ++t) {
                 // S_t is free once its rows sit in registers; where P is written over S,
-                // only once P V of this step has consumed it
-                if (C::kSepP) named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
-                else w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
+                // only once P V of this step has consumed it.  In a shared S region the last
+                // occupant is the other tile (its step j for tile 0, its step j+1 for tile 1),
+                // or, where the block has one tile, that tile's own step j.  s_free[t] counts
+                // the loads of tile t in step order, and a tile can be at most one load ahead
+                // of the issuer, so the step's parity names the phase.
+                if (C::kSharedS) {
+                    if (ntiles == 1) w.wait(smem_u32(&bars.s_free[0]), j & 1, kWaitSFree);
+                    else if (t == 0) w.wait(smem_u32(&bars.s_free[1]), j & 1, kWaitSFree);
+                    else w.wait(smem_u32(&bars.s_free[0]), (j + 1) & 1, kWaitSFree);
+                } else if (C::kSepP) {
+                    named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
+                } else {
+                    w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
+                }
                 tc_fence_after_sync();
                 issue_qk(t, sk);
             }
@@ -539,7 +567,15 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 uint32_t s[kKeys];
                 tmem_ld_cols<kKeys>(tS, s);
                 tmem_wait_ld_cols<kKeys>(s);
-                if (C::kSepP && j + 1 < nkv) {
+                if (C::kSharedS) {
+                    // the region goes to the other tile's Q K^T of this step (from tile 0) or
+                    // to the next step's (from tile 1, or from a tile that is alone)
+                    if (j + 1 < nkv || (t == 0 && ntiles == 2)) {
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
+                    }
+                } else if (C::kSepP && j + 1 < nkv) {
                     // S may be overwritten by the next Q K^T from here on
                     tc_fence_before_sync();
                     named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
