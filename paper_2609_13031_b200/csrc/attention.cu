@@ -16,10 +16,9 @@
 // the next Q K^T of its tile can run underneath the softmax, and writes the
 // probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 / fp16 in
 // the 16-bit path) to its own tensor-memory region, from where it is the A operand
-// of O_t += P_t V.  Where 512 columns cannot hold a separate P (bf16, d = 128),
-// P is written over S and Q K^T waits for P V instead.  In the FP8 d = 128 path the
-// two tiles take turns in one S region (S | P0 P0' | P1 P1' | O0 | O1), which leaves
-// room for 128-key steps and two P buffers per tile.
+// of O_t += P_t V.  At d = 128 the two tiles take turns in one S region
+// (S | P0 | P1 | O0 | O1), which leaves room for 128-key steps, a separate P and, in
+// the FP8 path, two P buffers per tile.
 //
 // Scale placement (FP8 path): x = (alpha * s_q * s_k * log2 e) * S feeds exp2;
 // the V scale and 1/rowsum are applied to O in the epilogue.
@@ -67,15 +66,15 @@ struct Cfg {
     static constexpr int kBoxBytes = kRowBytes > 128 ? 128 : kRowBytes;  // swizzle span
     static constexpr int kBoxes = kRowBytes / kBoxBytes;        // TMA boxes per tile
     static constexpr int kBoxCols = kBoxBytes / kES;
-    static constexpr bool kSepP = !(kD == 128 && !kFp8);        // P in its own TMEM region
     static constexpr int kKeys = 128;                           // keys per step
-    // FP8, d = 128: tensor memory has no room for two 128-column S tiles next to O and P, so
-    // the two query tiles take turns in ONE S region: a tile's scores sit there only from its
+    // d = 128: tensor memory has no room for two 128-column S tiles next to O and P, so the
+    // two query tiles take turns in ONE S region: a tile's scores sit there only from its
     // Q K^T until its softmax warps have loaded them into registers (a small part of a step),
     // and the tiles run about half a step apart anyway.  The Q K^T of one tile waits for the
-    // other tile's load instead of for its own.  (96-key steps with two S regions, the layout
-    // before this one, cost 3.6 % more time; 128-key steps with P written over S 6 % more.)
-    static constexpr bool kSharedS = kFp8 && kD == 128;
+    // other tile's load instead of for its own.  (Layouts before this one: FP8 with 96-key
+    // steps and two S regions, 3.6 % more time; P written over S, where Q K^T has to wait
+    // for P V: the 16-bit kernel took 10 % more time and 20 % more cycles that way.)
+    static constexpr bool kSharedS = kD == 128;
     static constexpr int kQTileBytes = kTileM * kRowBytes;
     static constexpr int kKVTileBytes = kKeys * kRowBytes;
     static constexpr int kUmmaK = 32 / kES;                     // elements per MMA K step
@@ -88,18 +87,17 @@ struct Cfg {
     // TMEM columns: S_t (one region for both tiles where shared), then O_t at 256 + t*kD, P_t
     // wherever 32-column-aligned room is left
     static constexpr uint32_t kColS0 = 0, kColS1 = kSharedS ? 0 : kKeys, kColO = 256;
-    static constexpr uint32_t kColP0 = !kSepP ? kColS0 : (kD == 128 ? 128u : 384u);
-    static constexpr uint32_t kColP1 = !kSepP ? kColS1 : (kD == 128 ? 192u : 384u + 64u);
+    static constexpr uint32_t kColP0 = kD == 128 ? 128u : 384u;
+    static constexpr uint32_t kColP1 = kD == 128 ? 192u : 384u + 64u;
     // Where tensor memory has room, P alternates between two buffers per tile (the second
     // kPCols columns after the first), so that writing P of one step never waits for the
     // P V of the step before.
     static constexpr int kPBufs = kFp8 ? 2 : 1;
     static constexpr bool kLateRescale = kD == 128;             // O rescale at the end of the step
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
-    static constexpr int kPolyPer16 = kFp8 ? 4 : (kD == 128 ? 8 : 2);
-    static_assert(kPBufs == 1 || (kSepP && 2 * kPCols <= 64), "TMEM layout");
-    static_assert(!kSepP || kD == 64 || (kSharedS && kKeys <= 128 && kPCols <= 32), "TMEM layout");
-    static_assert(!kSepP || kD == 128 || kPCols <= 64, "TMEM layout");
+    static constexpr int kPolyPer16 = kFp8 ? 4 : 2;
+    static_assert(kPBufs * kPCols <= 64, "TMEM layout: 64 columns of P per tile");
+    static_assert(kSharedS ? kKeys <= 128 : 2 * kKeys <= 256, "TMEM layout: S below column 256 (d = 64) or 128");
     static constexpr size_t kSmemBytes = (size_t)2 * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
 };
 
@@ -488,8 +486,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             const int sk = (j + 1) % C::kStages;
             w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
             for (int t = 0; t < ntiles; ++t) {
-                // S_t is free once its rows sit in registers; where P is written over S,
-                // only once P V of this step has consumed it.  In a shared S region the last
+                // S_t is free once its rows sit in registers.  In a shared S region the last
                 // occupant is the other tile (its step j for tile 0, its step j+1 for tile 1),
                 // or, where the block has one tile, that tile's own step j.  s_free[t] counts
                 // the loads of tile t in step order, and a tile can be at most one load ahead
@@ -498,10 +495,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     if (ntiles == 1) w.wait(smem_u32(&bars.s_free[0]), j & 1, kWaitSFree);
                     else if (t == 0) w.wait(smem_u32(&bars.s_free[1]), j & 1, kWaitSFree);
                     else w.wait(smem_u32(&bars.s_free[0]), (j + 1) & 1, kWaitSFree);
-                } else if (C::kSepP) {
-                    named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
                 } else {
-                    w.wait(smem_u32(&bars.p_free[t]), j & 1, kWaitPFree);
+                    named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
                 }
                 tc_fence_after_sync();
                 issue_qk(t, sk);
@@ -575,7 +570,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
                     }
-                } else if (C::kSepP && j + 1 < nkv) {
+                } else if (j + 1 < nkv) {
                     // S may be overwritten by the next Q K^T from here on
                     tc_fence_before_sync();
                     named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
@@ -600,7 +595,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 // the keys seen so far maps to 2^lift.
                 const float m_new = fmaxf(m, m_tile);
                 // P V of the previous step must be done before O is rescaled or P rewritten
-                bool pv_done = !(C::kSepP && j > 0);
+                bool pv_done = j == 0;
                 if (C::kPBufs == 1 && !pv_done && !w.dead) {
                     // ask now, use the answer a chunk of exponentials later: the usual case
                     // (P V long done) then costs no stall in the middle of the chunk
