@@ -153,8 +153,6 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
         wait(s_in, e_start);
         wait(s_cmp, e_start);
         wait(s_out, e_start);
-        // ... and its kernels after those of the host step before it on the device
-        if (g_last_compute[dev] != nullptr) cu(cudaStreamWaitEvent(s_cmp, g_last_compute[dev], 0));
         char* base = static_cast<char*>(device_scratch);
         // the small head of each set's workspace (status words, counters, accumulators) starts at zero
         const size_t ws_head = fp8attn_workspace_bytes(1, p.chunk_heads, 0, 0, d);
@@ -179,6 +177,9 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
             record(e_in[c], s_in);
             // ---- quantize + attention ----
             wait(s_cmp, e_in[c]);
+            // ... and the kernels of this call after those of the host step before it on the device
+            // (behind this call's first copies: on a caller's stream they are ahead of the wait)
+            if (c == 0 && g_last_compute[dev] != nullptr) cu(cudaStreamWaitEvent(s_cmp, g_last_compute[dev], 0));
             if (c >= p.sets) wait(s_cmp, e_o[c - p.sets]);   // the set's outputs have left
             float* scales = reinterpret_cast<float*>(set + p.off_scales);
             void* t16 = n_test > 0 ? set + p.off_t : nullptr;
