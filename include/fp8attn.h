@@ -186,7 +186,8 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
  * outputs of bf16attn_icl_forward_ex (which then is an fp16 kernel).
  *
  * FP8ATTN_SPLIT_TAIL balances the last, partly filled round of the launch.  The
- * grid is one CTA per 256 query rows of a head; when the number of CTAs is not
+ * grid is one CTA per 256 query rows of a head (per 384 at d = 64 in launches of
+ * eight rounds and more, which the split does not apply to); when the number of CTAs is not
  * a multiple of the number of SMs, the CTAs left over after the last full
  * round would run alone on a fraction of the GPU.  With this flag each of them
  * is replaced by up to 16 CTAs that share its query rows and divide the train

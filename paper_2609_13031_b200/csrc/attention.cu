@@ -1,24 +1,22 @@
 // Fused ICL attention for sm_100a: train->train and test->train in one launch.
 //
-// One CTA owns up to 256 query rows (two 128-row tiles) of one (b,h) and walks
-// over all train keys in steps of kKeys keys.  Warp roles:
-//   warps 0-3   softmax of query tile 0, one row per thread
-//   warps 4-7   softmax of query tile 1
-//   warp  8     issues the Q K^T tcgen05.mma of both tiles (one elected lane)
-//   warp  9     TMA producer for Q, K and V tiles
-//   warps 10-11 issue the P V tcgen05.mma of tile 0 and tile 1
+// One CTA owns the query rows of up to T 128-row tiles of one (b,h) (T = 3 at d = 64, 2 at
+// d = 128) and walks over all train keys in steps of kKeys keys.  Warp roles:
+//   warps 4t .. 4t+3   softmax of query tile t, one row per thread
+//   warp  4T           issues the Q K^T tcgen05.mma of all tiles (one elected lane)
+//   warp  4T+1         TMA producer for Q, K and V tiles
+//   warps 4T+2, 4T+3   issue the P V tcgen05.mma of tiles {0, 2} and {1}
 // Q K^T and P V are issued from different warps because a single warp cannot
 // issue tcgen05 instructions of this size fast enough to keep the tensor core fed.
 // A share of the exponentials (Cfg::kPolyPer16 pairs of every 16) is computed by a
 // polynomial on the FMA pipe instead of the MUFU.
-// Tensor memory (512 columns) holds S0 | S1 | (P0 | P1) | O0 | O1.  A softmax
-// thread pulls its whole score row into registers, releases S at once so that
-// the next Q K^T of its tile can run underneath the softmax, and writes the
-// probability tile P_t (e4m3 with the row maximum lifted to 2^8, or bf16 / fp16 in
-// the 16-bit path) to its own tensor-memory region, from where it is the A operand
-// of O_t += P_t V.  At d = 128 the two tiles take turns in one S region
-// (S | P0 | P1 | O0 | O1), which leaves room for 128-key steps, a separate P and, in
-// the FP8 path, two P buffers per tile.
+// Tensor memory (512 columns) holds S | P_0 .. P_(T-1) | O_0 .. O_(T-1): the tiles take
+// turns in ONE S region.  A softmax thread pulls its whole score row into registers
+// and gives S up at once, so that the Q K^T of the next tile in the rotation can run
+// underneath the softmax, and writes the probability tile P_t (e4m3 with the row
+// maximum lifted to 2^8, or bf16 / fp16 in the 16-bit path) to its own tensor-memory
+// region (two alternating buffers in the FP8 path), from where it is the A operand of
+// O_t += P_t V.
 //
 // Scale placement (FP8 path): x = (alpha * s_q * s_k * log2 e) * S feeds exp2;
 // the V scale and 1/rowsum are applied to O in the epilogue.
@@ -34,17 +32,24 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileM = 128;           // query rows per tile
-constexpr int kSoftmaxWarps = 8;
-constexpr int kQkWarp = 8, kTmaWarp = 9, kPvWarp0 = 10;
-constexpr int kNumThreads = 12 * 32;
-// Register budgets after setmaxnreg.  The CTA's register pool is what it was
-// launched with (384 threads x 168 registers); setmaxnreg.inc waits in hardware
-// until the pool can serve it, so the budgets must fit in it.
-constexpr int kLaunchRegs = 168;
-constexpr int kRegsSoftmax = 224;
+// Query tiles per CTA (kT): two, or at d = 64 three for launches of many rounds (tensor memory
+// holds 512 columns and every tile's O takes d of them).  Three tiles put a third softmax warp
+// on every scheduler, at the price of a smaller register budget per thread (96-key steps) and
+// coarser blocks (384 rows), which small grids pay for in their last round.  Warps: four
+// softmax warps per tile, then the Q K^T issuer, the TMA producer and two P V issuers (tiles
+// {0, 2} and {1}).
+template <int kT> constexpr int kRowsPerBlock = kT * kTileM;
+static_assert(kRowsPerBlock<2> == 256, "split_scratch_bytes() in api.cu sizes the scratch for blocks of 256 rows");
+template <int kT> constexpr int kNumThreads = (4 * kT + 4) * 32;
+// Register budgets after setmaxnreg.  The CTA's register pool is what it was launched with
+// (threads x registers at launch, as ptxas reports them for the launch bound);
+// setmaxnreg.inc waits in hardware until the pool can serve it, so the budgets must fit in it.
+template <int kT> constexpr int kLaunchRegs = kT == 3 ? 128 : 168;
+template <int kT> constexpr int kRegsSoftmax = kT == 3 ? 152 : 224;
 constexpr int kRegsOther = 56;
-static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= kNumThreads * kLaunchRegs,
-              "setmaxnreg budgets exceed the CTA's register pool");
+template <int kT> constexpr bool kRegsFit =
+    4 * kT * 32 * kRegsSoftmax<kT> + 4 * 32 * kRegsOther <= kNumThreads<kT> * kLaunchRegs<kT>;
+static_assert(kRegsFit<2> && kRegsFit<3>, "setmaxnreg budgets exceed the CTA's register pool");
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxSplits = 16;        // key ranges a split query block is divided into, at most
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
@@ -59,22 +64,18 @@ enum : uint32_t {
 // call is IEEE fp16 instead of bf16: the outputs of both kernels, and the operands and P
 // of the 16-bit kernel.  (A run-time switch for the FP8 kernel's output type cost 4 % at
 // d = 64 through register allocation, hence a template parameter.)
-template <bool kFp8, int kD, bool kHalf = false>
+template <bool kFp8, int kD, bool kHalf, int kT>
 struct Cfg {
+    static_assert(kT == 2 || (kT == 3 && kD == 64), "tiles per CTA");
     static constexpr int kES = kFp8 ? 1 : 2;                    // element bytes
     static constexpr int kRowBytes = kD * kES;
     static constexpr int kBoxBytes = kRowBytes > 128 ? 128 : kRowBytes;  // swizzle span
     static constexpr int kBoxes = kRowBytes / kBoxBytes;        // TMA boxes per tile
     static constexpr int kBoxCols = kBoxBytes / kES;
-    static constexpr int kKeys = 128;                           // keys per step
-    // d = 128: tensor memory has no room for two 128-column S tiles next to O and P, so the
-    // two query tiles take turns in ONE S region: a tile's scores sit there only from its
-    // Q K^T until its softmax warps have loaded them into registers (a small part of a step),
-    // and the tiles run about half a step apart anyway.  The Q K^T of one tile waits for the
-    // other tile's load instead of for its own.  (Layouts before this one: FP8 with 96-key
-    // steps and two S regions, 3.6 % more time; P written over S, where Q K^T has to wait
-    // for P V: the 16-bit kernel took 10 % more time and 20 % more cycles that way.)
-    static constexpr bool kSharedS = kD == 128;
+    static constexpr int kTiles = kT;
+    // keys per step: a softmax thread holds the scores of one row of a step in registers,
+    // 128 of them in a budget of 224 registers, 96 in a budget of 152
+    static constexpr int kKeys = kTiles == 3 ? 96 : 128;
     static constexpr int kQTileBytes = kTileM * kRowBytes;
     static constexpr int kKVTileBytes = kKeys * kRowBytes;
     static constexpr int kUmmaK = 32 / kES;                     // elements per MMA K step
@@ -84,27 +85,34 @@ struct Cfg {
     static constexpr uint32_t kIdescQK = idesc(kFmt, kFmt, false, false, kTileM, kKeys);
     static constexpr uint32_t kIdescPV = idesc(kFmt, kFmt, false, true, kTileM, kD);
     static constexpr int kPCols = kKeys * kES / 4;              // TMEM columns of a P tile
-    // TMEM columns: S_t (one region for both tiles where shared), then O_t at 256 + t*kD, P_t
-    // wherever 32-column-aligned room is left
-    static constexpr uint32_t kColS0 = 0, kColS1 = kSharedS ? 0 : kKeys, kColO = 256;
-    static constexpr uint32_t kColP0 = kD == 128 ? 128u : 384u;
-    static constexpr uint32_t kColP1 = kD == 128 ? 192u : 384u + 64u;
-    // Where tensor memory has room, P alternates between two buffers per tile (the second
-    // kPCols columns after the first), so that writing P of one step never waits for the
-    // P V of the step before.
+    // Tensor memory (512 columns): one S region that the query tiles of the CTA take turns in,
+    // the P tiles behind it, and O_t at 256 + t*kD.  A tile's scores sit in S only from its
+    // Q K^T until its softmax warps have loaded them into registers (a small part of a step),
+    // and the tiles run a fraction of a step apart anyway; the Q K^T of a tile waits for the
+    // load of the tile before it in the rotation.  Two tiles: S | P0 | P1 | O0 | O1 (128,
+    // 2 x 64, 2 x kD columns); three tiles (d = 64): S | P0 | P1 | P2 | - | O0 | O1 | O2 (96,
+    // 3 x 48, 3 x 64).
+    // (Layouts before this one, d = 128: FP8 with 96-key steps and an S region per tile,
+    // 3.6 % more time; P written over S, where Q K^T has to wait for P V: the 16-bit kernel
+    // took 10 % more time and 20 % more cycles that way.)
+    static constexpr uint32_t kColS = 0, kColO = 256;
+    static constexpr uint32_t kColP0 = kKeys, kPStride = kKeys / 2;   // P_t at kColP0 + t*kPStride
+    // FP8: P alternates between two buffers per tile (the second kPCols columns after the
+    // first), so that writing P of one step never waits for the P V of the step before.
     static constexpr int kPBufs = kFp8 ? 2 : 1;
-    static constexpr bool kLateRescale = kD == 128;             // O rescale at the end of the step
+    // O is rescaled at the end of the step, when the score registers are free
+    static constexpr bool kLateRescale = true;
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
-    static constexpr int kPolyPer16 = kFp8 ? 4 : 2;
-    static_assert(kPBufs * kPCols <= 64, "TMEM layout: 64 columns of P per tile");
-    static_assert(kSharedS ? kKeys <= 128 : 2 * kKeys <= 256, "TMEM layout: S below column 256 (d = 64) or 128");
-    static constexpr size_t kSmemBytes = (size_t)2 * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
+    static constexpr int kPolyPer16 = (kFp8 && kD == 128) ? 4 : 2;
+    static_assert(kPBufs * kPCols <= (int)kPStride, "TMEM layout: P tiles overlap");
+    static_assert(kColP0 + kTiles * kPStride <= kColO && kColO + kTiles * kD <= 512, "TMEM layout");
+    static constexpr size_t kSmemBytes = (size_t)kTiles * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
 };
 
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], p_free[2], o_full[2], s_free[2];
+    uint64_t s_full[3], p_free[3], o_full[3], s_free[3];
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -294,10 +302,9 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) 
     else tmem_st_x32(taddr, r);
 }
 
-// Named barriers (hardware-blocking, no polling), one of each per query tile t:
-//   kSFreeBarrier0 + t  "S_t is in registers"        softmax warps -> Q K^T issuer
+// Named barrier (hardware-blocking, no polling), one per query tile t:
 //   kPFullBarrier0 + t  "P_t is in tensor memory"    softmax warps -> P V issuer of tile t
-constexpr uint32_t kSFreeBarrier0 = 1, kPFullBarrier0 = 3;
+constexpr uint32_t kPFullBarrier0 = 1;
 constexpr uint32_t kSignalThreads = 128 + 32;   // one tile's softmax threads + the issuer warp
 
 // floats per row of a partial result: kD values of O, c*m, l, and padding to 16 bytes
@@ -307,28 +314,30 @@ struct KernelArgs {
     const float* scale_q; const float* scale_k; const float* scale_v;
     void* out_train; void* out_test;
     int64_t n_train, n_test;
-    int blocks_train, blocks_test;   // 256-row query blocks per head
+    int blocks_train, blocks_test;   // query blocks (one CTA's rows) per head
     int heads;                       // H, to find head 0 of a table
     int test_kv_head0;               // test rows read K, V and their scales from head 0 of their table
     // Tail split: the query blocks from full_blocks on (the part of the grid that would
     // fill less than one CTA per SM) are each run by `splits` CTAs over disjoint key ranges;
     // those CTAs write unnormalised partial results to `partial`, combined afterwards.
     int full_blocks, splits;
-    float* partial;                  // [unit][split][256 rows][kD + 4] fp32: O, c*m, l, pad
+    float* partial;                  // [unit][split][rows of a block][kD + 4] fp32: O, c*m, l, pad
     float softmax_scale;
     uint32_t* status;
 };
 
 // kSplit: this launch runs the split query blocks (see KernelArgs); kept out of the main
 // instantiation, whose softmax warps have no register to spare for the extra indices.
-template <bool kFp8, int kD, bool kHalf, bool kSplit>
-__global__ void __launch_bounds__(kNumThreads, 1)
+template <bool kFp8, int kD, bool kHalf, int kT, bool kSplit>
+__global__ void __launch_bounds__(kNumThreads<kT>, 1)
 icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                      const __grid_constant__ CUtensorMap map_q_test,
                      const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const KernelArgs args) {
-    using C = Cfg<kFp8, kD, kHalf>;
+    using C = Cfg<kFp8, kD, kHalf, kT>;
     constexpr int kKeys = C::kKeys;
+    constexpr int kQkWarp = 4 * C::kTiles, kTmaWarp = kQkWarp + 1, kPvWarp0 = kQkWarp + 2;
+    constexpr int kRows = kRowsPerBlock<kT>;       // query rows per CTA
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ uint32_t tmem_slot;
@@ -337,7 +346,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + 2 * C::kQTileBytes;
+    const uint32_t sK = sQ + C::kTiles * C::kQTileBytes;
     const uint32_t sV = sK + C::kStages * C::kKVTileBytes;
 
     // ---- which query block is this CTA's ----
@@ -349,8 +358,8 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     const int blk = vblk % blocks_per_head;
     const bool is_test = blk >= args.blocks_train;
     const int64_t q_rows = is_test ? args.n_test : args.n_train;
-    const int64_t row0 = (int64_t)(is_test ? blk - args.blocks_train : blk) * (2 * kTileM);
-    const int ntiles = (q_rows - row0 > kTileM) ? 2 : 1;
+    const int64_t row0 = (int64_t)(is_test ? blk - args.blocks_train : blk) * kRows;
+    const int ntiles = (int)min((int64_t)C::kTiles, (q_rows - row0 + kTileM - 1) / kTileM);
     const int64_t n_keys = args.n_train;
     // this CTA's key steps: [j0, j0 + nkv) of the nkv_all steps over the train keys
     const int nkv_all = (int)((n_keys + kKeys - 1) / kKeys);
@@ -380,7 +389,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             mbar_init(smem_u32(&bars.v_full[s]), 1);
             mbar_init(smem_u32(&bars.v_empty[s]), ntiles);   // one commit per P V issuer
         }
-        for (int t = 0; t < 2; ++t) {
+        for (int t = 0; t < C::kTiles; ++t) {
             mbar_init(smem_u32(&bars.s_full[t]), 1);
             mbar_init(smem_u32(&bars.p_free[t]), 1);
             mbar_init(smem_u32(&bars.o_full[t]), 1);
@@ -455,7 +464,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         auto issue_qk = [&](int t, int stage) {
             const uint64_t a0 = dQ + (uint64_t)((t * C::kQTileBytes) >> 4);
             const uint64_t b0 = dK + (uint64_t)((stage * C::kKVTileBytes) >> 4);
-            const uint32_t d = tmem + (t ? C::kColS1 : C::kColS0);
+            const uint32_t d = tmem + C::kColS;
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kD / C::kUmmaK; ++kk) {
@@ -473,9 +482,9 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         w.wait(smem_u32(&bars.k_full[0]), 0, kWaitKFull);
         tc_fence_after_sync();
         for (int t = 0; t < ntiles; ++t) {
-            if (C::kSharedS && t == 1) {
-                // the shared S region is tile 0's until its rows sit in registers
-                w.wait(smem_u32(&bars.s_free[0]), 0, kWaitSFree);
+            if (t > 0) {
+                // the S region is the tile's before this one until its rows sit in registers
+                w.wait(smem_u32(&bars.s_free[t - 1]), 0, kWaitSFree);
                 tc_fence_after_sync();
             }
             issue_qk(t, 0);
@@ -486,18 +495,13 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
             const int sk = (j + 1) % C::kStages;
             w.wait(smem_u32(&bars.k_full[sk]), ((j + 1) / C::kStages) & 1, kWaitKFull);
             for (int t = 0; t < ntiles; ++t) {
-                // S_t is free once its rows sit in registers.  In a shared S region the last
-                // occupant is the other tile (its step j for tile 0, its step j+1 for tile 1),
-                // or, where the block has one tile, that tile's own step j.  s_free[t] counts
-                // the loads of tile t in step order, and a tile can be at most one load ahead
-                // of the issuer, so the step's parity names the phase.
-                if (C::kSharedS) {
-                    if (ntiles == 1) w.wait(smem_u32(&bars.s_free[0]), j & 1, kWaitSFree);
-                    else if (t == 0) w.wait(smem_u32(&bars.s_free[1]), j & 1, kWaitSFree);
-                    else w.wait(smem_u32(&bars.s_free[0]), (j + 1) & 1, kWaitSFree);
-                } else {
-                    named_barrier_sync(kSFreeBarrier0 + t, kSignalThreads);
-                }
+                // The S region is free once its last occupant's rows sit in registers: that
+                // is the tile before this one in the rotation (step j+1 of tile t-1, or step j
+                // of the block's last tile for tile 0).  s_free[t] counts the loads of tile t
+                // in step order, and a tile can be at most one load ahead of the issuer, so
+                // the step's parity names the phase.
+                if (t == 0) w.wait(smem_u32(&bars.s_free[ntiles - 1]), j & 1, kWaitSFree);
+                else w.wait(smem_u32(&bars.s_free[t - 1]), (j + 1) & 1, kWaitSFree);
                 tc_fence_after_sync();
                 issue_qk(t, sk);
             }
@@ -506,14 +510,16 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
     } else if (warp >= kPvWarp0) {
         setmaxnreg_dec<kRegsOther>();
-        // ========================= P V issuer of one query tile =========================
-        const int t = warp - kPvWarp0;
-        if (t < ntiles) {
-            const uint64_t dV = smem_desc(sV, kKeys * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
-            const uint32_t d = tmem + C::kColO + t * kD;
-            const uint32_t a = tmem + (t ? C::kColP1 : C::kColP0);
-            for (int j = 0; j < nkv; ++j) {
-                const int sv = j % C::kStages;
+        // ============ P V issuers: the first takes tiles 0 and 2, the second tile 1 ============
+        // (the tiles' P become ready in the order of the rotation, so the tiles of one issuer
+        // never wait for each other)
+        const int pw = warp - kPvWarp0;
+        const uint64_t dV = smem_desc(sV, kKeys * C::kBoxBytes, 8 * C::kBoxBytes, C::kSwizzle);
+        for (int j = 0; j < nkv; ++j) {
+            const int sv = j % C::kStages;
+            for (int t = pw; t < ntiles; t += 2) {
+                const uint32_t d = tmem + C::kColO + t * kD;
+                const uint32_t a = tmem + C::kColP0 + (uint32_t)t * C::kPStride;
                 w.wait(smem_u32(&bars.v_full[sv]), (j / C::kStages) & 1, kWaitVFull);
                 named_barrier_sync(kPFullBarrier0 + t, kSignalThreads);
                 tc_fence_after_sync();
@@ -535,13 +541,13 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
     } else {
         // ========================= softmax + epilogue =========================
-        setmaxnreg_inc<kRegsSoftmax>();
+        setmaxnreg_inc<kRegsSoftmax<kT>>();
         const int t = warp >> 2;                       // query tile
         if (t < ntiles) {
             const int row_in_tile = (warp & 3) * 32 + lane;
             const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + lane_addr + (t ? C::kColS1 : C::kColS0);
-            const uint32_t tP = tmem + lane_addr + (t ? C::kColP1 : C::kColP0);
+            const uint32_t tS = tmem + lane_addr + C::kColS;
+            const uint32_t tP = tmem + lane_addr + C::kColP0 + (uint32_t)t * C::kPStride;
             const uint32_t tO = tmem + lane_addr + C::kColO + t * kD;
             float c = (args.softmax_scale > 0.f ? args.softmax_scale : rsqrtf((float)kD)) *
                       1.4426950408889634f;
@@ -562,18 +568,12 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 uint32_t s[kKeys];
                 tmem_ld_cols<kKeys>(tS, s);
                 tmem_wait_ld_cols<kKeys>(s);
-                if (C::kSharedS) {
-                    // the region goes to the other tile's Q K^T of this step (from tile 0) or
-                    // to the next step's (from tile 1, or from a tile that is alone)
-                    if (j + 1 < nkv || (t == 0 && ntiles == 2)) {
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
-                    }
-                } else if (j + 1 < nkv) {
-                    // S may be overwritten by the next Q K^T from here on
+                // the S region goes to the next tile's Q K^T of this step or, from the block's
+                // last tile, to tile 0's of the next step
+                if (j + 1 < nkv || t < ntiles - 1) {
                     tc_fence_before_sync();
-                    named_barrier_arrive(kSFreeBarrier0 + t, kSignalThreads);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.s_free[t]));
                 }
                 const int valid = (int)min((int64_t)kKeys, n_keys - (int64_t)(j0 + j) * kKeys);
                 if (valid < kKeys) {
@@ -724,7 +724,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                 // partial result of this key range: unnormalised O, the reference maximum in
                 // exp2 units and the row sum; the combine kernel weighs and normalises
                 float* dst = args.partial +
-                             ((size_t)((vblk - args.full_blocks) * nsplit + split) * (2 * kTileM) +
+                             ((size_t)((vblk - args.full_blocks) * nsplit + split) * kRowsPerBlock<kT> +
                               (size_t)(t * kTileM + row_in_tile)) * kPartialStride<kD>;
 #pragma unroll
                 for (int q = 0; q < kD / 32; ++q) {
@@ -788,25 +788,25 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
 // Combines the partial results of the split query blocks: with M = max_s c*m_s,
 // out = s_v * sum_s 2^(c*m_s - M) O_s / sum_s 2^(c*m_s - M) l_s.  One thread per row and
 // eight output columns.
-template <int kD>
+template <int kD, int kT>
 __global__ void __launch_bounds__(256)
 combine_split_kernel(const KernelArgs args, int units, int out_half, int fp8) {
     const int per_row = kD / 8;
     const int64_t tid = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    const int64_t unit = tid / (2 * kTileM * per_row);
+    const int64_t unit = tid / (kRowsPerBlock<kT> * per_row);
     if (unit >= units) return;
-    const int r = (int)(tid / per_row) % (2 * kTileM);
+    const int r = (int)(tid / per_row) % kRowsPerBlock<kT>;
     const int g = (int)(tid % per_row);
     const int blocks_per_head = args.blocks_train + args.blocks_test;
     const int vblk = args.full_blocks + (int)unit;
     const int bh = vblk / blocks_per_head, blk = vblk % blocks_per_head;
     const bool is_test = blk >= args.blocks_train;
     const int64_t q_rows = is_test ? args.n_test : args.n_train;
-    const int64_t row = (int64_t)(is_test ? blk - args.blocks_train : blk) * (2 * kTileM) + r;
+    const int64_t row = (int64_t)(is_test ? blk - args.blocks_train : blk) * kRowsPerBlock<kT> + r;
     if (row >= q_rows) return;
     const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
-    const float* base = args.partial + ((size_t)unit * args.splits * (2 * kTileM) + r) * kPartialStride<kD>;
-    const size_t split_stride = (size_t)(2 * kTileM) * kPartialStride<kD>;
+    const float* base = args.partial + ((size_t)unit * args.splits * kRowsPerBlock<kT> + r) * kPartialStride<kD>;
+    const size_t split_stride = (size_t)kRowsPerBlock<kT> * kPartialStride<kD>;
     float mmax = -INFINITY;
     for (int s = 0; s < args.splits; ++s) mmax = fmaxf(mmax, base[s * split_stride + kD]);
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -836,9 +836,9 @@ combine_split_kernel(const KernelArgs args, int units, int out_half, int fp8) {
     *reinterpret_cast<uint4*>(out + g * 8) = v;
 }
 
-template <bool kFp8, int kD, bool kHalf>
+template <bool kFp8, int kD, bool kHalf, int kT>
 int launch(const AttnParams& p, cudaStream_t stream) {
-    using C = Cfg<kFp8, kD, kHalf>;
+    using C = Cfg<kFp8, kD, kHalf, kT>;
     const int64_t heads = (int64_t)p.B * p.H;
     const bool test_only = (p.flags & FP8ATTN_TEST_ROWS_ONLY) != 0;
     CUtensorMap mq_train, mq_test, mk, mv;
@@ -859,8 +859,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     a.scale_q = p.scale_q; a.scale_k = p.scale_k; a.scale_v = p.scale_v;
     a.out_train = p.out_train; a.out_test = p.out_test;
     a.n_train = p.n_train; a.n_test = p.n_test;
-    a.blocks_train = test_only ? 0 : (int)((p.n_train + 2 * kTileM - 1) / (2 * kTileM));
-    a.blocks_test = (int)((p.n_test + 2 * kTileM - 1) / (2 * kTileM));
+    a.blocks_train = test_only ? 0 : (int)((p.n_train + kRowsPerBlock<kT> - 1) / kRowsPerBlock<kT>);
+    a.blocks_test = (int)((p.n_test + kRowsPerBlock<kT> - 1) / kRowsPerBlock<kT>);
     a.softmax_scale = p.softmax_scale;
     a.heads = p.H;
     a.test_kv_head0 = (p.flags & FP8ATTN_TEST_ROWS_USE_KV_HEAD0) ? 1 : 0;
@@ -875,7 +875,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     a.splits = 1;
     a.partial = nullptr;
     int units = 0;
-    if ((p.flags & FP8ATTN_SPLIT_TAIL) && p.partial != nullptr) {
+    // (three-tile launches have at least eight rounds, where the split does not pay)
+    if (kT == 2 && (p.flags & FP8ATTN_SPLIT_TAIL) && p.partial != nullptr) {
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
             return FP8ATTN_ERR_CUDA;
@@ -889,7 +890,7 @@ int launch(const AttnParams& p, cudaStream_t stream) {
             int64_t splits = sms / left;
             if (splits > steps / 4) splits = steps / 4;
             if (splits > kMaxSplits) splits = kMaxSplits;
-            const size_t per_split = (size_t)left * 2 * kTileM * kPartialStride<kD> * sizeof(float);
+            const size_t per_split = (size_t)left * kRowsPerBlock<kT> * kPartialStride<kD> * sizeof(float);
             while (splits >= 2 && per_split * (size_t)splits > p.partial_bytes) --splits;
             if (splits >= 2) {
                 a.full_blocks = (int)full;
@@ -899,8 +900,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
             }
         }
     }
-    auto kern = icl_attention_kernel<kFp8, kD, kHalf, false>;
-    auto kern_split = icl_attention_kernel<kFp8, kD, kHalf, true>;
+    auto kern = icl_attention_kernel<kFp8, kD, kHalf, kT, false>;
+    auto kern_split = icl_attention_kernel<kFp8, kD, kHalf, 2, true>;
     // The opt-in to large dynamic shared memory is per device and per context; it is set on
     // every call (a cached flag would go stale when the context is destroyed).
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes) !=
@@ -915,7 +916,7 @@ int launch(const AttnParams& p, cudaStream_t stream) {
         // The combine kernel is an ordinary launch behind the main grid, and the main grid
         // executes griddepcontrol.wait before it exits, so its completion implies that of the
         // split grid and the visibility of the partial results.
-        kern_split<<<(unsigned)(units * a.splits), kNumThreads, C::kSmemBytes, stream>>>(mq_train, mq_test,
+        kern_split<<<(unsigned)(units * a.splits), kNumThreads<kT>, C::kSmemBytes, stream>>>(mq_train, mq_test,
                                                                                       mk, mv, a);
         if (cudaGetLastError() != cudaSuccess) return FP8ATTN_ERR_CUDA;
         count_launch();
@@ -923,7 +924,7 @@ int launch(const AttnParams& p, cudaStream_t stream) {
     if (a.full_blocks > 0) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)a.full_blocks);
-        cfg.blockDim = dim3(kNumThreads);
+        cfg.blockDim = dim3(kNumThreads<kT>);
         cfg.dynamicSmemBytes = C::kSmemBytes;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -936,8 +937,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
         count_launch();
     }
     if (units > 0) {
-        const int64_t threads = (int64_t)units * 2 * kTileM * (kD / 8);
-        combine_split_kernel<kD><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
+        const int64_t threads = (int64_t)units * kRowsPerBlock<kT> * (kD / 8);
+        combine_split_kernel<kD, 2><<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
             a, units, kHalf ? 1 : 0, kFp8 ? 1 : 0);
         count_launch();
     }
@@ -966,14 +967,30 @@ int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
 }
 
+// d = 64: three tiles per CTA where the grid of 384-row blocks still fills the SMs at least
+// eight times over (there the last, partly filled round no longer matters, and neither does
+// the tail split); two tiles per CTA for smaller launches.
+template <bool kFp8, bool kHalf>
+int launch_d64(const AttnParams& p, cudaStream_t stream) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return FP8ATTN_ERR_CUDA;
+    const int64_t rows3 = kRowsPerBlock<3>;
+    const int64_t blocks = ((p.flags & FP8ATTN_TEST_ROWS_ONLY) ? 0 : (p.n_train + rows3 - 1) / rows3) +
+                           (p.n_test + rows3 - 1) / rows3;
+    if ((int64_t)p.B * p.H * blocks >= 8 * (int64_t)sms) return launch<kFp8, 64, kHalf, 3>(p, stream);
+    return launch<kFp8, 64, kHalf, 2>(p, stream);
+}
+
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {
     const bool half = (p.flags & FP8ATTN_IO_FP16) != 0;
     if (fp8) {
-        if (half) return p.d == 64 ? launch<true, 64, true>(p, stream) : launch<true, 128, true>(p, stream);
-        return p.d == 64 ? launch<true, 64, false>(p, stream) : launch<true, 128, false>(p, stream);
+        if (half) return p.d == 64 ? launch_d64<true, true>(p, stream) : launch<true, 128, true, 2>(p, stream);
+        return p.d == 64 ? launch_d64<true, false>(p, stream) : launch<true, 128, false, 2>(p, stream);
     }
-    if (half) return p.d == 64 ? launch<false, 64, true>(p, stream) : launch<false, 128, true>(p, stream);
-    return p.d == 64 ? launch<false, 64, false>(p, stream) : launch<false, 128, false>(p, stream);
+    if (half) return p.d == 64 ? launch_d64<false, true>(p, stream) : launch<false, 128, true, 2>(p, stream);
+    return p.d == 64 ? launch_d64<false, false>(p, stream) : launch<false, 128, false, 2>(p, stream);
 }
 
 }  // namespace fp8attn
