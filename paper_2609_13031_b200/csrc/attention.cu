@@ -103,7 +103,7 @@ struct Cfg {
     // O is rescaled at the end of the step, when the score registers are free
     static constexpr bool kLateRescale = true;
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
-    static constexpr int kPolyPer16 = (kFp8 && kD == 128) ? 4 : 2;
+    static constexpr int kPolyPer16 = kFp8 ? (kT == 3 ? 2 : 4) : 2;
     static_assert(kPBufs * kPCols <= (int)kPStride, "TMEM layout: P tiles overlap");
     static_assert(kColP0 + kTiles * kPStride <= kColO && kColO + kTiles * kD <= 512, "TMEM layout");
     static constexpr size_t kSmemBytes = (size_t)kTiles * kQTileBytes + (size_t)2 * kStages * kKVTileBytes + 1024;
