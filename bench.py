@@ -28,9 +28,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 NOMINAL_FP8_OVER_BF16 = 2.0           # dense tensor peak ratio (4.5 / 2.25 PFLOP/s)
-# exponentials per clock per SM: the 16-lane MUFU alone, and with a quarter of them on the FMA pipe
+# exponentials per clock per SM: the 16-lane MUFU alone; with a share f of them on the FMA pipe
+# the limit is 16 / (1 - f)
 SOFTMAX_MUFU_PER_CLK_SM = 16.0
-SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM = 16.0 / 0.75
+
+
+def fma_share_of_exponentials(w, sms: int) -> float:
+    """Share of the FP8 kernel's exponentials that it evaluates by a polynomial on the FMA pipe:
+    a quarter, or an eighth in the three-tile launches (d = 64, at least eight rounds of
+    384-row blocks)."""
+    blocks3 = w.B * w.H * (-(-w.n_train // 384) + -(-w.n_test // 384))
+    return 0.125 if (w.d == 64 and blocks3 >= 8 * sms) else 0.25
 
 
 def ncu_dram_traffic(workload: str):
@@ -498,18 +506,20 @@ def main():
         peak_fp8_burst = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops"]
         quant_bytes = w.B * w.H * w.d * (5 * 3 * w.n_train + 3 * w.n_test)
         # secondary roofline: the exponential path.  One exponential per score; the MUFU
-        # evaluates 16 per clock per SM, and with a quarter of them on the FMA pipe the
-        # limit is 21.3.  Clock = the median SM clock sampled during the timed steps.
+        # evaluates 16 per clock per SM, and with the kernel's share of them on the FMA pipe
+        # the limit is 16 / (1 - share).  Clock = the median SM clock sampled during the timed steps.
         sms = torch.cuda.get_device_properties(local).multi_processor_count
         scores = float(w.B) * w.H * w.n_train * (w.n_train + w.n_test)
         softmax = None
         if clocks.get("sm_mhz"):
             per_clk_sm = scores / (ms_attn * 1e-3) / (sms * clocks["sm_mhz"] * 1e6)
+            share = fma_share_of_exponentials(w, sms)
             softmax = {"scores_per_clk_per_sm": per_clk_sm,
                        "mufu_only_peak": SOFTMAX_MUFU_PER_CLK_SM,
                        "frac_of_mufu_only": per_clk_sm / SOFTMAX_MUFU_PER_CLK_SM,
-                       "quarter_on_fma_peak": SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM,
-                       "frac": per_clk_sm / SOFTMAX_WITH_FMA_SHARE_PER_CLK_SM,
+                       "fma_share": share,
+                       "with_fma_share_peak": SOFTMAX_MUFU_PER_CLK_SM / (1.0 - share),
+                       "frac": per_clk_sm * (1.0 - share) / SOFTMAX_MUFU_PER_CLK_SM,
                        "clock_mhz": clocks["sm_mhz"], "sms": sms}
         traffic = ncu_dram_traffic(w.name)
         line = {
