@@ -233,6 +233,14 @@ int bf16attn_icl_forward_ex(const void* q_train, const void* q_test, const void*
 #define FP8ATTN_GATE_TRAIN_ROWS 8192
 int fp8attn_gate_use_fp8(int64_t n_train);
 
+/* Informational, host only (the paper has no counterpart): the number of query rows that
+ * one CTA of the forward calls takes for a call of these sizes and flags on the current
+ * device: 256 (two 128-row tiles), or 384 (three) at d = 64 when the grid of 384-row
+ * blocks fills the SMs at least eight times over.  Without a device the SM count of a
+ * B200 (148) is assumed.  0 for unsupported sizes.  Results do not depend on it beyond the
+ * order of the online softmax (steps of 128 or 96 keys). */
+int fp8attn_attention_rows_per_cta(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags);
+
 /* Seeded Gaussian perturbation of Q, K or V (paper appendix, Eq. 3: the noise
  * experiment that replaces quantization by an explicit perturbation):
  *

@@ -26,7 +26,7 @@ EXPORTS = (
     "fp8attn_quantize_qkv", "fp8attn_quantize_qkv_ex", "fp8attn_perturb",
     "fp8attn_selftest_wait_timeout", "fp8attn_quantize_ex",
     "fp8attn_icl_step_host", "fp8attn_host_step_scratch_bytes", "fp8attn_host_step_chunks",
-    "fp8attn_host_step_status",
+    "fp8attn_host_step_status", "fp8attn_attention_rows_per_cta",
 )
 # flags of fp8attn_quantize_ex / fp8attn_quantize_qkv_ex
 QUERY_SCALE_FROM_ALL_ROWS = 1
@@ -104,6 +104,8 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_status_string.argtypes = [i32]
     lib.fp8attn_launch_count.restype = ctypes.c_uint64
     lib.fp8attn_launch_count.argtypes = []
+    lib.fp8attn_attention_rows_per_cta.restype = i32
+    lib.fp8attn_attention_rows_per_cta.argtypes = [i32, i32, i64, i64, i32, u32]
     lib.fp8attn_host_step_scratch_bytes.restype = sz
     lib.fp8attn_host_step_scratch_bytes.argtypes = [i32, i32, i64, i64, i32, u32]
     lib.fp8attn_host_step_chunks.restype = i32
@@ -249,6 +251,11 @@ def selftest_wait_timeout(workspace: torch.Tensor, limit_us: int = 1000) -> None
     """fp8attn_selftest_wait_timeout: make one bounded device wait expire on purpose."""
     rc = load().fp8attn_selftest_wait_timeout(_ptr(workspace), workspace.numel(), int(limit_us), _stream())
     _check("fp8attn_selftest_wait_timeout", rc)
+
+
+def attention_rows_per_cta(B: int, H: int, n_train: int, n_test: int, d: int, flags: int = 0) -> int:
+    """fp8attn_attention_rows_per_cta: 256 or 384 query rows per CTA for a call of these sizes."""
+    return int(load().fp8attn_attention_rows_per_cta(B, H, n_train, n_test, d, int(flags)))
 
 
 def gate_use_fp8(n_train: int) -> bool:

@@ -231,6 +231,16 @@ int fp8attn_selftest_wait_timeout(void* workspace, size_t workspace_bytes_, uint
 
 int fp8attn_gate_use_fp8(int64_t n_train) { return n_train > FP8ATTN_GATE_TRAIN_ROWS ? 1 : 0; }
 
+int fp8attn_attention_rows_per_cta(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags) {
+    if (B <= 0 || H <= 0 || n_train < 0 || n_test < 0 || (d != 64 && d != 128)) return 0;
+    // without a device to ask (a host without a GPU): the SM count of a B200
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    return fp8attn::attention_rows_per_cta(B, H, n_train, n_test, d, flags, sms);
+}
+
 size_t fp8attn_workspace_bytes(int B, int H, int64_t n_train, int64_t, int d) {
     if (B <= 0 || H <= 0) return 0;
     // with the size of an attention call: room for the tail split's partial results as well

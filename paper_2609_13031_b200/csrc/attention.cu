@@ -976,11 +976,17 @@ int launch_d64(const AttnParams& p, cudaStream_t stream) {
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return FP8ATTN_ERR_CUDA;
-    const int64_t rows3 = kRowsPerBlock<3>;
-    const int64_t blocks = ((p.flags & FP8ATTN_TEST_ROWS_ONLY) ? 0 : (p.n_train + rows3 - 1) / rows3) +
-                           (p.n_test + rows3 - 1) / rows3;
-    if ((int64_t)p.B * p.H * blocks >= 8 * (int64_t)sms) return launch<kFp8, 64, kHalf, 3>(p, stream);
+    if (attention_rows_per_cta(p.B, p.H, p.n_train, p.n_test, 64, p.flags, sms) == kRowsPerBlock<3>)
+        return launch<kFp8, 64, kHalf, 3>(p, stream);
     return launch<kFp8, 64, kHalf, 2>(p, stream);
+}
+
+int attention_rows_per_cta(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags, int sms) {
+    if (d != 64) return kRowsPerBlock<2>;
+    const int64_t rows3 = kRowsPerBlock<3>;
+    const int64_t blocks = ((flags & FP8ATTN_TEST_ROWS_ONLY) ? 0 : (n_train + rows3 - 1) / rows3) +
+                           (n_test + rows3 - 1) / rows3;
+    return (int64_t)B * H * blocks >= 8 * (int64_t)sms ? kRowsPerBlock<3> : kRowsPerBlock<2>;
 }
 
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream) {

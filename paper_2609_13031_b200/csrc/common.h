@@ -73,6 +73,9 @@ struct AttnParams {
     size_t partial_bytes;
 };
 int launch_icl_attention(const AttnParams& p, bool fp8, cudaStream_t stream);
+// Query rows per CTA that a forward call of these sizes uses on a device with `sms` SMs: 256, or
+// 384 at d = 64 where the grid of 384-row blocks fills the SMs at least eight times over.
+int attention_rows_per_cta(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags, int sms);
 int launch_wait_timeout_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
 
 }  // namespace fp8attn
