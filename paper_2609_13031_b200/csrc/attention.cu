@@ -369,9 +369,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     // grouped-query variant: every test query head attends to the first K/V head of its table
     const int bh_kv = (is_test && args.test_kv_head0) ? (bh / args.heads) * args.heads : bh;
 
-    // the main launch does not depend on this one: let it start as soon as SMs are free
-    if (kSplit) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
     // A device error recorded earlier (and not yet read back by the host) is sticky:
     // nothing runs until fp8attn_last_device_status() has cleared it.
     // One thread reads it for the whole CTA, so that either every warp leaves or none does
@@ -775,14 +772,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
-    // Launched behind the split grid with programmatic stream serialization, this grid
-    // completes only after that one has (and its writes are visible): the combine kernel,
-    // ordered behind this grid, may then read the split grid's partial results.  The wait
-    // comes after the tensor memory has been given back, so that a CTA never waits for another
-    // grid while it holds an allocation that a CTA of that grid could be blocked on.  (With
-    // 168 registers x 384 threads one CTA fills an SM's register file, so two CTAs do not
-    // share an SM today; the order keeps that from becoming a requirement.)
-    if (!kSplit) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Combines the partial results of the split query blocks: with M = max_s c*m_s,
@@ -910,12 +899,11 @@ int launch(const AttnParams& p, cudaStream_t stream) {
                                            (int)C::kSmemBytes) != cudaSuccess))
         return FP8ATTN_ERR_CUDA;
     if (units > 0) {
-        // The split blocks go first and release their dependents at once, and the main launch
-        // is allowed to start while they run (programmatic dependent launch): the two grids
-        // are independent, so the SMs the short split CTAs leave go straight to main CTAs.
-        // The combine kernel is an ordinary launch behind the main grid, and the main grid
-        // executes griddepcontrol.wait before it exits, so its completion implies that of the
-        // split grid and the visibility of the partial results.
+        // The split blocks go first; the main grid and the combine kernel follow in stream
+        // order.  (Releasing the main grid early behind the split grid by programmatic dependent
+        // launch gained 1-2.5 % on launches of one to three rounds, but made the main grid's CTAs
+        // wait for the split grid before they exit, the only wait of the library that no
+        // time limit bounds.)
         kern_split<<<(unsigned)(units * a.splits), kNumThreads<kT>, C::kSmemBytes, stream>>>(mq_train, mq_test,
                                                                                       mk, mv, a);
         if (cudaGetLastError() != cudaSuccess) return FP8ATTN_ERR_CUDA;
@@ -927,11 +915,8 @@ int launch(const AttnParams& p, cudaStream_t stream) {
         cfg.blockDim = dim3(kNumThreads<kT>);
         cfg.dynamicSmemBytes = C::kSmemBytes;
         cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = units > 0 ? 1 : 0;
+        cfg.attrs = nullptr;
+        cfg.numAttrs = 0;
         if (cudaLaunchKernelEx(&cfg, kern, mq_train, mq_test, mk, mv, a) != cudaSuccess)
             return FP8ATTN_ERR_CUDA;
         count_launch();
