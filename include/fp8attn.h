@@ -202,10 +202,6 @@ int bf16attn_icl_forward(const void* q_train, const void* q_test, const void* k,
  * rows take the split path depends on the sizes of the call, so a row's result
  * is no longer bit-identical across calls with different n_test.
  *
- * Calls with this flag belong on one stream: run from two streams at the same time they
- * stalled a B200 (the main grid is released early behind the split grid and waits for it
- * before it exits; the cause of the stall was not established).
- *
  * Unknown flag bits return FP8ATTN_ERR_INVALID_ARG.  flags = 0 is the plain call.
  */
 #define FP8ATTN_TEST_ROWS_USE_KV_HEAD0 1u
@@ -324,10 +320,7 @@ int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int
  * in `cuda_stream`; `cuda_stream` continues after the last copy-out), so the host buffers
  * must stay valid, and the outputs are complete, once `cuda_stream` has been synchronised.
  * Calls made on different streams (each with its own scratch and host buffers) may be in
- * flight together: their copies overlap the other call's kernels.  Their kernels do not
- * overlap: the library orders the kernels of host steps on a device in the order of the
- * calls (attention launches with FP8ATTN_SPLIT_TAIL from two streams at once stalled the
- * GPU when it was tried).
+ * flight together: the copies and kernels of one overlap those of the other.
  * The library allocates no device memory here either; it creates and releases three
  * streams and a few events per call.  fp8attn_host_step_status synchronises `cuda_stream`
  * and returns the device status of the call's workspaces (inside the scratch), like

@@ -6,8 +6,6 @@
 // between chunks.  Everything is enqueued; the host is not synchronised.
 #include <cuda_runtime.h>
 
-#include <mutex>
-
 #include "common.h"
 
 namespace fp8attn {
@@ -17,15 +15,6 @@ constexpr int kMaxChunks = 8;
 constexpr int64_t kPipelineMinBytes = 32ll << 20;   // 16-bit input bytes below which one chunk is used
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
-
-// The kernels of two host steps never overlap on a GPU: the compute stream of every call waits
-// for the last kernel of the call before it on the same device, whatever stream that was made
-// on.  (Two pipelined calls running their attention launches side by side from different streams
-// stalled the GPU when it was tried.)  The copies of a call made on another stream are free to
-// overlap those kernels, which is all that two calls in flight can gain.
-constexpr int kMaxDevices = 64;
-std::mutex g_order_mutex;
-cudaEvent_t g_last_compute[kMaxDevices] = {};
 
 struct Plan {
     int heads;            // B*H
@@ -110,7 +99,9 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
         device_scratch_bytes < p.set_bytes * (size_t)p.sets)
         return FP8ATTN_ERR_WORKSPACE;
     cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
-    const uint32_t qflags = (flags & FP8ATTN_HOST_FP16) ? FP8ATTN_INPUT_FP16 : 0u;
+    // the two-launch quantizer: host steps of different streams may share the GPU, and the blocks
+    // of the one-launch form wait for one another
+    const uint32_t qflags = FP8ATTN_QKV_TWO_LAUNCHES | ((flags & FP8ATTN_HOST_FP16) ? FP8ATTN_INPUT_FP16 : 0u);
     const uint32_t fflags = FP8ATTN_SPLIT_TAIL | ((flags & FP8ATTN_HOST_FP16) ? FP8ATTN_IO_FP16 : 0u);
 
     // streams and events of this call; destroying them at the end only marks them for release
@@ -143,12 +134,8 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
     auto record = [&](cudaEvent_t e, cudaStream_t s) { if (own_streams) cu(cudaEventRecord(e, s)); };
     auto wait = [&](cudaStream_t s, cudaEvent_t e) { if (own_streams) cu(cudaStreamWaitEvent(s, e, 0)); };
 
-    int dev = 0;
-    if (rc == FP8ATTN_OK && (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)) rc = FP8ATTN_ERR_CUDA;
-    // one call at a time enqueues, so that the order of the calls on the GPU is the order of the calls
-    std::lock_guard<std::mutex> lock(g_order_mutex);
     if (rc == FP8ATTN_OK) {
-        // everything of this call comes after what the caller's stream holds so far ...
+        // everything of this call comes after what the caller's stream holds so far
         record(e_start, user);
         wait(s_in, e_start);
         wait(s_cmp, e_start);
@@ -177,9 +164,6 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
             record(e_in[c], s_in);
             // ---- quantize + attention ----
             wait(s_cmp, e_in[c]);
-            // ... and the kernels of this call after those of the host step before it on the device
-            // (behind this call's first copies: on a caller's stream they are ahead of the wait)
-            if (c == 0 && g_last_compute[dev] != nullptr) cu(cudaStreamWaitEvent(s_cmp, g_last_compute[dev], 0));
             if (c >= p.sets) wait(s_cmp, e_o[c - p.sets]);   // the set's outputs have left
             float* scales = reinterpret_cast<float*>(set + p.off_scales);
             void* t16 = n_test > 0 ? set + p.off_t : nullptr;
@@ -203,14 +187,6 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
                 cu(cudaMemcpyAsync(static_cast<char*>(out_test) + (size_t)h0 * head_test, set + p.off_ote, be,
                                    cudaMemcpyDeviceToHost, s_out));
             record(e_o[c], s_out);
-        }
-        // the last kernel of this call, for the next call's kernels to wait on
-        cudaEvent_t done = nullptr;
-        if (cu(cudaEventCreateWithFlags(&done, cudaEventDisableTiming)) && cu(cudaEventRecord(done, s_cmp))) {
-            if (g_last_compute[dev] != nullptr) cudaEventDestroy(g_last_compute[dev]);
-            g_last_compute[dev] = done;
-        } else if (done != nullptr) {
-            cudaEventDestroy(done);
         }
         // the caller's stream continues after all three
         cudaStream_t all[3] = {s_in, s_cmp, s_out};

@@ -121,8 +121,7 @@ def test_fp16_tensors():
 
 
 def test_calls_in_flight_on_two_streams():
-    # two calls, two streams, own scratch each: copies may overlap the other call's kernels; the
-    # library keeps the kernels of the two calls apart
+    # two calls, two streams, own scratch each: the copies and kernels of one overlap the other's
     w = dataclasses.replace(W.CONFIGS["C3"].scaled(8192, 1024), B=1, H=6)
     ga, gb = W.generate(w), W.generate(dataclasses.replace(w, seed=w.seed + 100))
     xa = {k: host16(v) for k, v in ga.items()}
