@@ -100,8 +100,6 @@ struct Cfg {
     // FP8: P alternates between two buffers per tile (the second kPCols columns after the
     // first), so that writing P of one step never waits for the P V of the step before.
     static constexpr int kPBufs = kFp8 ? 2 : 1;
-    // O is rescaled at the end of the step, when the score registers are free
-    static constexpr bool kLateRescale = true;
     // pairs of exponentials, out of every 16 pairs, that go to the FMA pipe (measured best)
     static constexpr int kPolyPer16 = kFp8 ? (kT == 3 ? 2 : 4) : 2;
     static_assert(kPBufs * kPCols <= (int)kPStride, "TMEM layout: P tiles overlap");
@@ -450,7 +448,7 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
         }
     } else if (warp == kQkWarp) {
         setmaxnreg_dec<kRegsOther>();
-        // ====================== Q K^T issuer (both query tiles) ======================
+        // ====================== Q K^T issuer (all query tiles) ======================
         // The whole warp walks the loop (waits included); one elected lane issues the
         // MMAs and commits.  Q K^T and P V are issued from different warps because one
         // warp cannot issue tcgen05 instructions fast enough to feed the tensor core
@@ -599,12 +597,10 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     pv_done = mbar_test_wait(smem_u32(&bars.p_free[t]), (j - 1) & 1);
                     tc_fence_after_sync();
                 }
-                // Where the maximum moved for some row of this warp, l is rescaled now.  O is
-                // rescaled now too (kLateRescale false), or at the end of the step: by then
-                // the score registers are free, so the O columns go through registers in
-                // pipelined halves instead of dependent 16-column round trips, and the P V
-                // that has to precede it is long done.  Measured: late wins at d = 128,
-                // early at d = 64.
+                // Where the maximum moved for some row of this warp, l is rescaled now and O at
+                // the end of the step: by then the score registers are free, so the O columns
+                // go through registers in pipelined 64-column halves instead of dependent
+                // 16-column round trips, and the P V that has to precede it is long done.
                 const bool rescale = j > 0 && __any_sync(0xffffffffu, m_new > m);
                 float f = 1.0f;
                 if (rescale) {
@@ -612,22 +608,6 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     const uint64_t ff = pack2(f, f);
                     l2a = mul2(l2a, ff);
                     l2b = mul2(l2b, ff);
-                    if (!C::kLateRescale) {
-                        if (!pv_done) {
-                            w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
-                            tc_fence_after_sync();
-                            pv_done = true;
-                        }
-#pragma unroll
-                        for (int q = 0; q < kD / 16; ++q) {
-                            uint32_t o[16];
-                            tmem_ld_x16(tO + q * 16, o);
-                            tmem_wait_ld_x16(o);
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                            tmem_st_x16(tO + q * 16, o);
-                        }
-                    }
                 }
                 m = m_new;
                 const float nb = lift - m * c;
@@ -683,9 +663,9 @@ icl_attention_kernel(const __grid_constant__ CUtensorMap map_q_train,
                     // That write comes after the next step's fence behind its wait for S.
                     w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                     pv_done = true;
-                    if (C::kLateRescale && rescale) tc_fence_after_sync();
+                    if (rescale) tc_fence_after_sync();
                 }
-                if (C::kLateRescale && rescale) {
+                if (rescale) {
                     if (!pv_done) {
                         w.wait(smem_u32(&bars.p_free[t]), (j - 1) & 1, kWaitPFree);
                         tc_fence_after_sync();
