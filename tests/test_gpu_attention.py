@@ -165,6 +165,11 @@ def test_bf16_c3_full_size_sampled():
     check_bf16_case(W.CONFIGS["C3"], n_sample=128)
 
 
+def test_bf16_c4_full_size_sampled():
+    # d = 64 at a size that takes the three-tile kernel
+    check_bf16_case(W.CONFIGS["C4"], n_sample=32)
+
+
 # ---- structure of the ICL layer -------------------------------------------------------
 
 def test_test_rows_are_batch_invariant_and_share_kv_with_train_rows():
