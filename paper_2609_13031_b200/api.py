@@ -27,6 +27,7 @@ EXPORTS = (
     "fp8attn_selftest_wait_timeout", "fp8attn_quantize_ex",
     "fp8attn_icl_step_host", "fp8attn_host_step_scratch_bytes", "fp8attn_host_step_chunks",
     "fp8attn_host_step_status", "fp8attn_attention_rows_per_cta",
+    "fp8attn_quantize_qkv_ordered", "fp8attn_reorder_rows",
 )
 # flags of fp8attn_quantize_ex / fp8attn_quantize_qkv_ex
 QUERY_SCALE_FROM_ALL_ROWS = 1
@@ -87,6 +88,11 @@ def load() -> ctypes.CDLL:
     lib.fp8attn_quantize_qkv_ex.restype = i32
     lib.fp8attn_quantize_qkv_ex.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
                                             vp, vp, vp, u32, vp, sz, vp]
+    lib.fp8attn_quantize_qkv_ordered.restype = i32
+    lib.fp8attn_quantize_qkv_ordered.argtypes = [vp, vp, vp, vp, i32, i32, i64, i64, i32, vp, vp, vp, vp,
+                                                 vp, vp, vp, vp, u32, vp, sz, vp]
+    lib.fp8attn_reorder_rows.restype = i32
+    lib.fp8attn_reorder_rows.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp]
     lib.fp8attn_perturb.restype = i32
     lib.fp8attn_perturb.argtypes = [vp, i32, i32, i64, i32, f32, ctypes.c_uint64, u32, vp, vp, vp, sz, vp]
     lib.fp8attn_selftest_wait_timeout.restype = i32
@@ -199,11 +205,13 @@ def quantize_noalloc(x: torch.Tensor, out: torch.Tensor, scale_out: torch.Tensor
     return out, scale_out
 
 
-def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
+def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0, order_keys: bool = False):
     """fp8attn_quantize_qkv: all four quantizations of one attention call in two
     launches.  Returns dict(q8, k8, v8, t8, sq, sk, sv); ``out`` may supply those
     tensors preallocated.  With SCALES_GIVEN, ``out`` must hold sq, sk, sv and they
-    are read instead of written (one launch)."""
+    are read instead of written (one launch).  ``order_keys``:
+    fp8attn_quantize_qkv_ordered, K8 and V8 come out with the keys of largest norm first and
+    the dict also holds ``key_dest`` (int32 [B,H,n_train], the row each key moved to)."""
     if flags & SCALES_GIVEN:
         assert out is not None and all(n in out for n in ("sq", "sk", "sv"))
     B, H, n_train, d = _dims(k)
@@ -223,13 +231,30 @@ def quantize_qkv(q_train, k, v, q_test, workspace, out=None, flags: int = 0):
     args = (_ptr(q_train), _ptr(k), _ptr(v), _ptr(q_test) if n_test else None, B, H, n_train, n_test, d,
             _ptr(o["q8"]), _ptr(o["k8"]), _ptr(o["v8"]), _ptr(o["t8"]) if n_test else None,
             _ptr(o["sq"]), _ptr(o["sk"]), _ptr(o["sv"]))
-    if flags:
+    if order_keys:
+        if "key_dest" not in o:
+            o["key_dest"] = torch.empty((B, H, n_train), dtype=torch.int32, device=dev)
+        rc = load().fp8attn_quantize_qkv_ordered(*args, _ptr(o["key_dest"]), int(flags), _ptr(workspace),
+                                                 workspace.numel(), _stream())
+        _check("fp8attn_quantize_qkv_ordered", rc)
+    elif flags:
         rc = load().fp8attn_quantize_qkv_ex(*args, int(flags), _ptr(workspace), workspace.numel(), _stream())
         _check("fp8attn_quantize_qkv_ex", rc)
     else:
         rc = load().fp8attn_quantize_qkv(*args, _ptr(workspace), workspace.numel(), _stream())
         _check("fp8attn_quantize_qkv", rc)
     return o
+
+
+def reorder_rows(x: torch.Tensor, dest: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """fp8attn_reorder_rows: out[b,h,dest[b,h,r],:] = x[b,h,r,:] for a 16-bit tensor."""
+    B, H, rows, d = _dims(x)
+    assert _is16(x) and dest.dtype == torch.int32 and dest.is_cuda and dest.is_contiguous() and dest.numel() == B * H * rows
+    if out is None:
+        out = torch.empty_like(x)
+    rc = load().fp8attn_reorder_rows(_ptr(x), B, H, rows, d, _ptr(dest), _ptr(out), _stream())
+    _check("fp8attn_reorder_rows", rc)
+    return out
 
 
 def perturb(x: torch.Tensor, epsilon: float, seed: int, stream_id: int, workspace: torch.Tensor,

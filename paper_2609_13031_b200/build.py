@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libfp8attn.so")
-SOURCES = ["api.cu", "quantize.cu", "attention.cu", "perturb.cu", "host_step.cu"]
+SOURCES = ["api.cu", "quantize.cu", "attention.cu", "perturb.cu", "host_step.cu", "key_order.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

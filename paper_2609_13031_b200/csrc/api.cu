@@ -122,10 +122,15 @@ int fp8attn_quantize_ex(const void* x_bf16, int B, int H, int64_t rows, int d, c
                            flags, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test, int B,
-                         int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
-                         void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k, float* scale_v,
-                         uint32_t flags, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// key_dest: NULL for the plain call; else the keys are ordered first and K, V written in that order
+int quantize_qkv_impl(const void* q_train, const void* k, const void* v, const void* q_test, int B,
+                      int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
+                      void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k, float* scale_v,
+                      int32_t* key_dest, uint32_t flags, void* workspace, size_t workspace_bytes_,
+                      void* cuda_stream) {
     int rc = check_shape(B, H, d);
     if (rc != FP8ATTN_OK) return rc;
     if (n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
@@ -146,11 +151,51 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
     if (rc != FP8ATTN_OK) return rc;
     uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
     char* ws = static_cast<char*>(workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (key_dest != nullptr) {
+        rc = launch_key_order(k, (int64_t)B * H, n_train, d, (flags & FP8ATTN_INPUT_FP16) != 0, key_dest, stream);
+        if (rc != FP8ATTN_OK) return rc;
+    }
     return launch_quantize_qkv(q_train, k, v, q_test, (int64_t)B * H, n_train * (int64_t)d,
                                n_test * (int64_t)d, q_train_fp8, k_fp8, v_fp8, q_test_fp8, scale_q, scale_k,
                                scale_v, amax, flags, reinterpret_cast<uint32_t*>(ws + kWsStatusOffset),
                                reinterpret_cast<uint32_t*>(ws + kWsCounterOffset),
-                               reinterpret_cast<float*>(ws + ws_partial_offset(B, H)),
+                               reinterpret_cast<float*>(ws + ws_partial_offset(B, H)), stream, key_dest, d);
+}
+}  // namespace
+
+extern "C" {
+
+int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, const void* q_test, int B,
+                         int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
+                         void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k, float* scale_v,
+                         uint32_t flags, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    return quantize_qkv_impl(q_train, k, v, q_test, B, H, n_train, n_test, d, q_train_fp8, k_fp8, v_fp8,
+                             q_test_fp8, scale_q, scale_k, scale_v, nullptr, flags, workspace, workspace_bytes_,
+                             cuda_stream);
+}
+
+int fp8attn_quantize_qkv_ordered(const void* q_train, const void* k, const void* v, const void* q_test, int B,
+                                 int H, int64_t n_train, int64_t n_test, int d, void* q_train_fp8, void* k_fp8,
+                                 void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
+                                 float* scale_v, int32_t* key_dest, uint32_t flags, void* workspace,
+                                 size_t workspace_bytes_, void* cuda_stream) {
+    if (!key_dest || !aligned(key_dest, 4)) return FP8ATTN_ERR_INVALID_ARG;
+    return quantize_qkv_impl(q_train, k, v, q_test, B, H, n_train, n_test, d, q_train_fp8, k_fp8, v_fp8,
+                             q_test_fp8, scale_q, scale_k, scale_v, key_dest, flags, workspace, workspace_bytes_,
+                             cuda_stream);
+}
+
+int fp8attn_reorder_rows(const void* x_16bit, int B, int H, int64_t rows, int d, const int32_t* dest,
+                         void* out_16bit, void* cuda_stream) {
+    int rc = check_shape(B, H, d);
+    if (rc != FP8ATTN_OK) return rc;
+    if (rows < 0) return FP8ATTN_ERR_INVALID_ARG;
+    if (rows > 0 && (!x_16bit || !dest || !out_16bit || x_16bit == out_16bit)) return FP8ATTN_ERR_INVALID_ARG;
+    if (!aligned(x_16bit, 16) || !aligned(out_16bit, 16) || !aligned(dest, 4)) return FP8ATTN_ERR_INVALID_ARG;
+    rc = check_device();
+    if (rc != FP8ATTN_OK) return rc;
+    return launch_reorder_rows(x_16bit, (int64_t)B * H, rows, d, dest, out_16bit,
                                static_cast<cudaStream_t>(cuda_stream));
 }
 

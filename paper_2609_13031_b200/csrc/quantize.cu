@@ -139,11 +139,15 @@ __device__ __forceinline__ uint32_t quant4(uint32_t w0, uint32_t w1, float s, co
 
 // One block's share of head blockIdx.y.  Each thread turns 32 B of 16-bit input into
 // 16 B of e4m3 per step.  pairs_per_head = elems_per_head / 16.
+// `row_dest` (NULL: none) sends the codes of row r of a head to row row_dest[r] of the output;
+// a row is 2^pairs_per_row_shift pairs.
 template <bool kHalf>
 __device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64_t pairs_per_head,
                                               const float* __restrict__ scale_in,
                                               const uint32_t* __restrict__ amax_bits,
-                                              uint4* __restrict__ out, float* __restrict__ scale_out) {
+                                              uint4* __restrict__ out, float* __restrict__ scale_out,
+                                              const int32_t* __restrict__ row_dest = nullptr,
+                                              int pairs_per_row_shift = 0) {
     float s;
     if (scale_in != nullptr) {
         s = scale_in[blockIdx.y];
@@ -183,7 +187,13 @@ __device__ __forceinline__ void quantize_body(const uint4* __restrict__ x, int64
             o.z = quant4<kHalf, false>(b.x, b.y, s, tab);
             o.w = quant4<kHalf, false>(b.z, b.w, s, tab);
         }
-        oh[i] = o;
+        int64_t dst = i;
+        if (row_dest != nullptr) {
+            const int64_t row = i >> pairs_per_row_shift;
+            dst = ((int64_t)row_dest[(int64_t)blockIdx.y * (pairs_per_head >> pairs_per_row_shift) + row]
+                   << pairs_per_row_shift) + (i - (row << pairs_per_row_shift));
+        }
+        oh[dst] = o;
     }
 }
 
@@ -205,6 +215,8 @@ struct QuantBatch {
     const uint32_t* amax_in[4];   // accumulators the scale is derived from
     uint32_t* amax_acc[4];        // accumulators this tensor's maximum goes to (NULL: none)
     float* scale_out[4];
+    const int32_t* row_dest[4];   // output row of every input row, per head (NULL: the same row)
+    int pairs_per_row_shift;      // log2(d / 16)
 };
 
 template <bool kHalf>
@@ -217,7 +229,8 @@ __global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch
 template <bool kHalf>
 __global__ void __launch_bounds__(kThreads) quantize_batch_kernel(const QuantBatch b) {
     const int z = blockIdx.z;
-    quantize_body<kHalf>(b.x[z], b.pairs_per_head[z], b.scale_in[z], b.amax_in[z], b.out[z], b.scale_out[z]);
+    quantize_body<kHalf>(b.x[z], b.pairs_per_head[z], b.scale_in[z], b.amax_in[z], b.out[z], b.scale_out[z],
+                         b.row_dest[z], b.pairs_per_row_shift);
 }
 
 
@@ -414,7 +427,8 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
                         float* scale_v, uint32_t* amax_bits, uint32_t flags, uint32_t* status,
-                        uint32_t* counters, float* partial, cudaStream_t stream) {
+                        uint32_t* counters, float* partial, cudaStream_t stream, const int32_t* key_dest,
+                        int d) {
     if (n_heads <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     QuantBatch b;
@@ -432,6 +446,8 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
         if (z == 3 && (flags & FP8ATTN_QUERY_SCALE_FROM_ALL_ROWS) && elems_test > 0) b.amax_acc[z] = amax_bits;
         b.scale_out[z] = scales[z];
         b.scale_in[z] = nullptr;
+        // a key order applies to K and V alike: the attention sums over keys
+        b.row_dest[z] = (z == 1 || z == 2) ? key_dest : nullptr;
         if (flags & FP8ATTN_SCALES_GIVEN) {
             // scales computed upstream: nothing to reduce, nothing to write back
             b.scale_in[z] = scales[z == 3 ? 0 : z];
@@ -439,13 +455,15 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
             b.amax_acc[z] = nullptr;
         }
     }
+    b.pairs_per_row_shift = d == 128 ? 3 : 2;
     const int tensors = elems_test > 0 ? 4 : 3;
     const int sms = sm_count();
     if (sms <= 0) return FP8ATTN_ERR_CUDA;
     const bool half = (flags & FP8ATTN_INPUT_FP16) != 0;
     // small call: one launch (maximum, grid barrier, conversion)
     const int64_t total_pairs = (3 * elems_train + elems_test) / 16 * n_heads;
-    if (!(flags & (FP8ATTN_SCALES_GIVEN | FP8ATTN_QKV_TWO_LAUNCHES)) && status != nullptr && total_pairs > 0 &&
+    if (!(flags & (FP8ATTN_SCALES_GIVEN | FP8ATTN_QKV_TWO_LAUNCHES)) && key_dest == nullptr && status != nullptr &&
+        total_pairs > 0 &&
         total_pairs * 32 <= kOneLaunchMaxBytes) {
         OneLaunchArgs a;
         a.b = b;
