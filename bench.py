@@ -249,6 +249,9 @@ def main():
                     help="run the named workload's recipe at this many train / test rows (profiling on small cases)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-rows", type=int, default=96, help="oracle sample: query rows per head and call")
+    ap.add_argument("--order-keys", default="auto", choices=["auto", "on", "off"],
+                    help="quantize with fp8attn_quantize_qkv_ordered (the keys of largest norm first); auto: "
+                         "from 32,768 train rows on, where its two extra launches cost under 1 %% of the step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-bf16", action="store_true")
     ap.add_argument("--no-fp8-gemm", action="store_true", help="skip the library FP8 GEMM rate (context figure)")
@@ -309,16 +312,28 @@ def main():
     host_out = {"o_tr": torch.empty(shape_tr, dtype=torch.bfloat16).pin_memory(),
                 "o_te": torch.empty(shape_te, dtype=torch.bfloat16).pin_memory()}
 
+    order_keys = args.order_keys == "on" or (args.order_keys == "auto" and w.n_train >= 32768)
+    if order_keys:
+        buf["key_dest"] = torch.empty((w.B, w.H, w.n_train), dtype=torch.int32, device="cuda")
+
     def quantize_all():
-        # all four quantizations (Q_train, K, V with their own scales; Q_test with Q_train's) in two launches
-        api.quantize_qkv(dev["q_train"], dev["k"], dev["v"], dev["q_test"], ws, out=buf)
+        # all four quantizations (Q_train, K, V with their own scales; Q_test with Q_train's) in two
+        # launches; with the key order, two more small launches and K8, V8 written in that order
+        api.quantize_qkv(dev["q_train"], dev["k"], dev["v"], dev["q_test"], ws, out=buf, order_keys=order_keys)
+
+    # the 16-bit comparison kernel runs on K, V in the same key order (reordered once, outside its timing)
+    twin_kv = {"k": dev["k"], "v": dev["v"]}
+    if order_keys and not args.no_bf16:
+        quantize_all()
+        twin_kv = {"k": api.reorder_rows(dev["k"], buf["key_dest"]), "v": api.reorder_rows(dev["v"], buf["key_dest"])}
+        torch.cuda.synchronize()
 
     def attention_fp8():
         api.icl_forward_fp8(buf["q8"], buf["t8"], buf["k8"], buf["v8"], buf["sq"], buf["sk"], buf["sv"],
                             ws, 0.0, out_train=buf["o_tr"], out_test=buf["o_te"], flags=fwd_flags)
 
     def attention_bf16():
-        api.icl_forward_bf16(dev["q_train"], dev["q_test"], dev["k"], dev["v"], ws, 0.0,
+        api.icl_forward_bf16(dev["q_train"], dev["q_test"], twin_kv["k"], twin_kv["v"], ws, 0.0,
                              out_train=buf["o_tr"], out_test=buf["o_te"], flags=fwd_flags)
 
     def sync_all():
@@ -418,17 +433,18 @@ def main():
     # heads.  Throughput: steps alternate between two streams (own device scratch and own host
     # result buffers each), so that the copies of one step overlap the kernels of the other.
     shape = (w.B, w.H, w.n_train, w.n_test, w.d)
+    host_flags = api.HOST_ORDER_KEYS if order_keys else 0
     n_slots = 2
     slots = []
     for _ in range(n_slots):
         slots.append({"stream": torch.cuda.Stream(),
-                      "scratch": torch.empty(api.host_step_scratch_bytes(*shape), dtype=torch.uint8, device="cuda"),
+                      "scratch": torch.empty(api.host_step_scratch_bytes(*shape, host_flags), dtype=torch.uint8, device="cuda"),
                       "o_tr": torch.empty_like(host_out["o_tr"]).pin_memory(),
                       "o_te": torch.empty_like(host_out["o_te"]).pin_memory()})
 
     def host_step(slot, flags=0, scratch=None):
         api.icl_step_host(host["q_train"], host["k"], host["v"], host["q_test"],
-                          slot["scratch"] if scratch is None else scratch, flags=flags,
+                          slot["scratch"] if scratch is None else scratch, flags=flags | host_flags,
                           out_train=slot["o_tr"], out_test=slot["o_te"])
 
     def e2e_run(n):
@@ -459,7 +475,7 @@ def main():
     sync_all()
     ms_e2e = max_over_ranks(a.elapsed_time(b)) / n_e2e
     for slot in slots:
-        st = api.host_step_status(slot["scratch"], *shape)
+        st = api.host_step_status(slot["scratch"], *shape, host_flags)
         if st != (0, 0):
             raise RuntimeError(f"device status after the end-to-end steps: {st}")
     h2d = sum(t.numel() * t.element_size() for t in host.values())
@@ -478,9 +494,10 @@ def main():
 
     ms_single = single_call(0, slots[0]["scratch"])
     slots[1]["scratch"] = None              # make room for the unpipelined call's larger scratch
-    one_chunk = torch.empty(api.host_step_scratch_bytes(*shape, api.HOST_ONE_CHUNK), dtype=torch.uint8, device="cuda")
+    one_chunk = torch.empty(api.host_step_scratch_bytes(*shape, api.HOST_ONE_CHUNK | host_flags), dtype=torch.uint8,
+                            device="cuda")
     ms_single_one_chunk = single_call(api.HOST_ONE_CHUNK, one_chunk)
-    n_chunks = api.host_step_chunks(*shape)
+    n_chunks = api.host_step_chunks(*shape, host_flags)
     del one_chunk
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N=1 only ----
@@ -528,7 +545,10 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
             "data": "synthetic",
             "config": {"workload": workload_label(w), "step": STEP_LABEL, "l2": l2_label(w)},
-            "impl_detail": {"calls": "fp8attn_quantize_qkv (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
+            "impl_detail": {"calls": ("fp8attn_quantize_qkv_ordered" if order_keys else "fp8attn_quantize_qkv") +
+                                     " (Q_train,K,V,Q_test) + fp8attn_icl_forward_ex (FP8ATTN_SPLIT_TAIL)",
+                            "key_order": ("the keys of largest norm first (chosen and applied inside the timed quantization; "
+                                          "the 16-bit comparison kernel runs on K, V in the same order)") if order_keys else "as given",
                             "preroll": "%d untimed steps (%.1f s) under the same load before the timed steps" % (pre_n, pre_s),
                             "replicas": world},
             "clocks": clocks,

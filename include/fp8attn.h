@@ -128,10 +128,11 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
  * counterpart: its kernel takes the keys as they come).  Attention sums over keys, so K and
  * V may be permuted together without changing the result; the order matters to the kernel
  * all the same, because every time a row's running maximum moves the accumulated output is
- * rescaled.  This call brings the keys of largest norm to the front (at least 256 per head:
+ * rescaled.  This call brings the keys of largest norm to the front (about 256 per head:
  * the rows whose squared norm, binned by exponent and four mantissa bits, lies at or above
- * the bin that the 256th largest falls in), where, for most queries, the row maximum then
- * settles in the first step; all other keys follow in their old order.
+ * the bin that the 32nd largest of every eighth row falls in), where, for most queries, the row maximum then
+ * settles in the first step; all other keys follow in their old order.  Where more than 2048
+ * rows of a head qualify (norms that single out no small group), that head keeps its order.
  *
  *   key_dest  out int32 [B,H,n_train] (device): the row that key r of head (b,h) was moved to,
  *             a permutation per head.  K8 and V8 are written in that order
@@ -341,7 +342,9 @@ int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int
  *                  fp8attn_host_step_scratch_bytes(...) bytes with the same sizes and flags;
  *                  its contents on entry do not matter
  *   flags          FP8ATTN_HOST_ONE_CHUNK (no pipeline), FP8ATTN_HOST_FP16 (all 16-bit tensors
- *                  are IEEE fp16); other bits: FP8ATTN_ERR_INVALID_ARG
+ *                  are IEEE fp16), FP8ATTN_HOST_ORDER_KEYS (quantize with
+ *                  fp8attn_quantize_qkv_ordered: the keys of largest norm first); other bits:
+ *                  FP8ATTN_ERR_INVALID_ARG
  *
  * The host buffers should be page-locked: copies from pageable memory are staged by the
  * CUDA runtime and do not overlap.  The call only enqueues work (after everything already
@@ -356,6 +359,7 @@ int fp8attn_quantize_noalloc(const void* x_bf16, int B, int H, int64_t rows, int
  * the call is cut into (0 for unsupported sizes, like the scratch size). */
 #define FP8ATTN_HOST_ONE_CHUNK 1u
 #define FP8ATTN_HOST_FP16 2u
+#define FP8ATTN_HOST_ORDER_KEYS 4u
 size_t fp8attn_host_step_scratch_bytes(int B, int H, int64_t n_train, int64_t n_test, int d,
                                        uint32_t flags);
 int fp8attn_host_step_chunks(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t flags);

@@ -43,6 +43,7 @@ GATE_TRAIN_ROWS = 8192
 # flags of fp8attn_icl_step_host
 HOST_ONE_CHUNK = 1
 HOST_FP16 = 2
+HOST_ORDER_KEYS = 4
 
 _lib = None
 

@@ -24,7 +24,7 @@ struct Plan {
     size_t in_train, in_test, out_train, out_test;   // bytes per chunk (16-bit tensors)
     size_t ws;            // workspace bytes per set
     // offsets inside one set
-    size_t off_ws, off_q, off_k, off_v, off_t, off_q8, off_k8, off_v8, off_t8, off_scales, off_otr, off_ote;
+    size_t off_ws, off_q, off_k, off_v, off_t, off_q8, off_k8, off_v8, off_t8, off_scales, off_otr, off_ote, off_order;
     size_t set_bytes;
 };
 
@@ -57,6 +57,7 @@ Plan make_plan(int B, int H, int64_t n_train, int64_t n_test, int d, uint32_t fl
     p.off_scales = take(3 * g * sizeof(float));
     p.off_otr = take(p.out_train);
     p.off_ote = take(p.out_test);
+    p.off_order = take((flags & FP8ATTN_HOST_ORDER_KEYS) ? g * (size_t)n_train * sizeof(int32_t) : 0);
     p.set_bytes = o;
     return p;
 }
@@ -88,7 +89,7 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
                                      float softmax_scale, uint32_t flags, void* out_train, void* out_test,
                                      void* device_scratch, size_t device_scratch_bytes, void* cuda_stream) {
     using namespace fp8attn;
-    if (flags & ~(FP8ATTN_HOST_ONE_CHUNK | FP8ATTN_HOST_FP16)) return FP8ATTN_ERR_INVALID_ARG;
+    if (flags & ~(FP8ATTN_HOST_ONE_CHUNK | FP8ATTN_HOST_FP16 | FP8ATTN_HOST_ORDER_KEYS)) return FP8ATTN_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || n_train < 1 || n_test < 0) return FP8ATTN_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return FP8ATTN_ERR_UNSUPPORTED;
     if (!args_ok(B, H, n_train, n_test, d)) return FP8ATTN_ERR_UNSUPPORTED;
@@ -169,9 +170,16 @@ extern "C" int fp8attn_icl_step_host(const void* q_train, const void* k, const v
             void* t16 = n_test > 0 ? set + p.off_t : nullptr;
             void* t8 = n_test > 0 ? set + p.off_t8 : nullptr;
             void* ote = n_test > 0 ? set + p.off_ote : nullptr;
-            int r = fp8attn_quantize_qkv_ex(set + p.off_q, set + p.off_k, set + p.off_v, t16, 1, g, n_train, n_test, d,
-                                            set + p.off_q8, set + p.off_k8, set + p.off_v8, t8, scales, scales + g,
-                                            scales + 2 * g, qflags, set + p.off_ws, p.ws, s_cmp);
+            int r = (flags & FP8ATTN_HOST_ORDER_KEYS)
+                        ? fp8attn_quantize_qkv_ordered(set + p.off_q, set + p.off_k, set + p.off_v, t16, 1, g, n_train,
+                                                       n_test, d, set + p.off_q8, set + p.off_k8, set + p.off_v8, t8,
+                                                       scales, scales + g, scales + 2 * g,
+                                                       reinterpret_cast<int32_t*>(set + p.off_order), qflags,
+                                                       set + p.off_ws, p.ws, s_cmp)
+                        : fp8attn_quantize_qkv_ex(set + p.off_q, set + p.off_k, set + p.off_v, t16, 1, g, n_train,
+                                                  n_test, d, set + p.off_q8, set + p.off_k8, set + p.off_v8, t8,
+                                                  scales, scales + g, scales + 2 * g, qflags, set + p.off_ws, p.ws,
+                                                  s_cmp);
             record(e_q[c], s_cmp);
             if (r == FP8ATTN_OK)
                 r = fp8attn_icl_forward_ex(set + p.off_q8, t8, set + p.off_k8, set + p.off_v8, scales, scales + g,

@@ -9,10 +9,11 @@
 // where they do not.)
 //
 //   key_norm_kernel   sum of squares of every key row (fp32), stored as its bit pattern in `dest`
-//   key_order_kernel  per head: histogram of the norms, the bin from which on at least
+//   key_order_kernel  per head: histogram of the norms of a sample, the bin from which on about
 //                     kFirstKeys rows lie, then a stable partition (rows at or above that bin
-//                     first, the others behind, both in their old order); `dest` becomes the
-//                     destination row of every key
+//                     first, the others behind, both in their old order; left alone where that
+//                     would be more than kMaxFirst rows); `dest` becomes the destination row of
+//                     every key
 //   reorder_rows_kernel  applies such a map to a 16-bit tensor (the FP8 path applies it while
 //                     it writes the codes)
 #include <cuda_bf16.h>
@@ -23,7 +24,7 @@
 namespace fp8attn {
 namespace {
 
-constexpr int kFirstKeys = 256;          // keys to bring to the front (two steps' worth)
+constexpr int kFirstKeys = 256;          // keys to bring to the front, about (two steps' worth)
 constexpr int kOrderThreads = 1024;
 constexpr int kBins = 4096;              // fp32 bit pattern >> 19: exponent and four mantissa bits
 
@@ -63,50 +64,103 @@ __global__ void __launch_bounds__(256) key_norm_kernel(const uint4* __restrict__
 }
 
 // One block per head.  On entry dest holds the rows' norms (fp32 bit patterns, non-negative, so
-// they order like unsigned integers); on exit the destination row of every row.
+// they order like unsigned integers); on exit the destination row of every row.  The rows at or
+// above the threshold bin are collected in a list (at most kMaxFirst: where more rows than that
+// share the leading bins, the norms single out no small group and the order is left alone),
+// the list is sorted, and every row finds its place by a binary search: a listed row goes to
+// its rank in the list, any other row r to r + (listed rows behind it).
+constexpr int kMaxFirst = 2048;
+constexpr int kSample = 8;
+
 __global__ void __launch_bounds__(kOrderThreads) key_order_kernel(int64_t rows, uint32_t* __restrict__ dest) {
     __shared__ uint32_t hist[kBins];
-    __shared__ uint32_t warp_sum[kOrderThreads / 32];
+    __shared__ uint32_t suffix[kOrderThreads];
+    __shared__ uint32_t list[kMaxFirst];
     __shared__ uint32_t threshold_bin, first_count;
     uint32_t* d = dest + (int64_t)blockIdx.x * rows;
-    for (int i = threadIdx.x; i < kBins; i += kOrderThreads) hist[i] = 0u;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < kBins; i += kOrderThreads) hist[i] = 0u;
+    if (tid == 0) first_count = 0u;
     __syncthreads();
-    for (int64_t i = threadIdx.x; i < rows; i += kOrderThreads) atomicAdd(&hist[d[i] >> 19], 1u);
+    // Histogram of a sample (every kSample-th row): the norms of a table crowd into few bins,
+    // and shared-memory atomics on them are what this kernel would otherwise spend its time on.
+    // The threshold then brings about kFirstKeys rows to the front instead of at least that many.
+    const int64_t sampled = (rows + kSample - 1) / kSample;
+    for (int64_t i = tid; i < sampled; i += kOrderThreads) atomicAdd(&hist[d[i * kSample] >> 19], 1u);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t count = 0;
-        int bin = kBins - 1;
-        for (; bin > 0; --bin) {
-            count += hist[bin];
-            if (count >= (uint32_t)kFirstKeys) break;
-        }
-        if (bin == 0) count += hist[0];
-        threshold_bin = (uint32_t)bin;
-        first_count = count;
+    constexpr uint32_t want = kFirstKeys / kSample;
+    // suffix[t] = rows in the bins from 4t on (kBins = 4 * kOrderThreads)
+    static_assert(kBins == 4 * kOrderThreads, "four bins per thread");
+    const uint32_t own = hist[4 * tid] + hist[4 * tid + 1] + hist[4 * tid + 2] + hist[4 * tid + 3];
+    suffix[tid] = own;
+    __syncthreads();
+    for (int o = 1; o < kOrderThreads; o <<= 1) {
+        const uint32_t add = tid + o < kOrderThreads ? suffix[tid + o] : 0u;
+        __syncthreads();
+        suffix[tid] += add;
+        __syncthreads();
     }
+    // the thread whose four bins contain the kFirstKeys-th largest row picks the bin
+    const uint32_t above = suffix[tid] - own;     // rows in the bins of the threads behind this one
+    if (above < want && suffix[tid] >= want) {
+        uint32_t count = above;
+        int bin = 4 * tid + 3;
+        for (;; --bin) {
+            count += hist[bin];
+            if (count >= want || bin == 4 * tid) break;
+        }
+        threshold_bin = (uint32_t)bin;
+    }
+    if (tid == 0 && suffix[0] < want) threshold_bin = 0u;   // fewer rows than that: all of them
     __syncthreads();
     const uint32_t thr = threshold_bin;
-    uint32_t first_off = 0, rest_off = first_count;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int64_t base = 0; base < rows; base += kOrderThreads) {
-        const int64_t i = base + threadIdx.x;
-        const bool in = i < rows;
-        const bool first = in && (d[i] >> 19) >= thr;
-        const uint32_t ballot = __ballot_sync(0xffffffffu, first);
-        const uint32_t before_in_warp = __popc(ballot & ((1u << lane) - 1u));
-        if (lane == 0) warp_sum[warp] = __popc(ballot);
-        __syncthreads();
-        uint32_t before = before_in_warp, total = 0;
-        for (int w = 0; w < kOrderThreads / 32; ++w) {
-            const uint32_t c = warp_sum[w];
-            if (w < warp) before += c;
-            total += c;
+    constexpr int kIlp = 8;   // independent loads in flight per thread: one block reads the whole head
+    for (int64_t base = tid; base < rows; base += (int64_t)kIlp * kOrderThreads) {
+        uint32_t v[kIlp];
+#pragma unroll
+        for (int u = 0; u < kIlp; ++u) {
+            const int64_t i = base + (int64_t)u * kOrderThreads;
+            v[u] = i < rows ? d[i] : 0xffffffffu;
         }
-        if (in) d[i] = first ? first_off + before : rest_off + ((uint32_t)threadIdx.x - before);
-        const uint32_t chunk = (uint32_t)min((int64_t)kOrderThreads, rows - base);
-        first_off += total;
-        rest_off += chunk - total;
-        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < kIlp; ++u) {
+            if (v[u] != 0xffffffffu && (v[u] >> 19) >= thr) {
+                const uint32_t pos = atomicAdd(&first_count, 1u);
+                if (pos < (uint32_t)kMaxFirst) list[pos] = (uint32_t)(base + (int64_t)u * kOrderThreads);
+            }
+        }
+    }
+    __syncthreads();
+    const uint32_t count = first_count;
+    if (count > (uint32_t)kMaxFirst || count == (uint32_t)rows) {
+        for (int64_t i = tid; i < rows; i += kOrderThreads) d[i] = (uint32_t)i;
+        return;
+    }
+    // bitonic sort of the list, padded with the largest value
+    for (int i = tid; i < kMaxFirst; i += kOrderThreads)
+        if ((uint32_t)i >= count) list[i] = 0xffffffffu;
+    __syncthreads();
+    for (int k = 2; k <= kMaxFirst; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < kMaxFirst; i += kOrderThreads) {
+                const int p = i ^ j;
+                if (p > i) {
+                    const uint32_t a = list[i], b = list[p];
+                    if (((i & k) == 0) ? a > b : a < b) { list[i] = b; list[p] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int64_t i = tid; i < rows; i += kOrderThreads) {
+        // listed rows below i (lower bound of i in the sorted list)
+        int lo = 0, hi = (int)count;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (list[mid] < (uint32_t)i) lo = mid + 1; else hi = mid;
+        }
+        const bool listed = lo < (int)count && list[lo] == (uint32_t)i;
+        d[i] = listed ? (uint32_t)lo : (uint32_t)i + (count - (uint32_t)lo);
     }
 }
 

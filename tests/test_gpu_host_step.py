@@ -108,6 +108,21 @@ def test_pipelined_chunks(H, expect_chunks, chunk_heads):
     check_against_oracle(w, g, p_tr, p_te, n_sample=24)
 
 
+def test_host_step_with_ordered_keys():
+    # FP8ATTN_HOST_ORDER_KEYS: every chunk quantizes with the keys of largest norm first; the
+    # result is attention over the same keys, so the oracle criteria are the same
+    w = dataclasses.replace(W.CONFIGS["C3"].scaled(8192, 1100), B=1, H=6)
+    assert api.host_step_chunks(*shape_of(w), api.HOST_ORDER_KEYS) == 6
+    assert api.host_step_scratch_bytes(*shape_of(w), api.HOST_ORDER_KEYS) > api.host_step_scratch_bytes(*shape_of(w))
+    g = W.generate(w)
+    _, o_tr, o_te = run_host_step(w, g, flags=api.HOST_ORDER_KEYS)
+    torch.cuda.synchronize()
+    check_against_oracle(w, g, o_tr, o_te, n_sample=24)
+    _, p_tr, p_te = run_host_step(w, g)
+    torch.cuda.synchronize()
+    assert not torch.equal(o_tr, p_tr)          # another order of the online softmax
+
+
 def test_fp16_tensors():
     w = dataclasses.replace(W.CONFIGS["C2"].scaled(900, 200), B=1, H=3)
     g = {k: np.ascontiguousarray(bf16_bits_to_f64(v).astype(np.float16)).view(np.uint16)
