@@ -153,7 +153,10 @@ int quantize_qkv_impl(const void* q_train, const void* k, const void* v, const v
     char* ws = static_cast<char*>(workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (key_dest != nullptr) {
-        rc = launch_key_order(k, (int64_t)B * H, n_train, d, (flags & FP8ATTN_INPUT_FP16) != 0, key_dest, stream);
+        // the key norms go through the K8 buffer (d bytes per key, of which four are used),
+        // which the conversion overwrites afterwards
+        rc = launch_key_order(k, (int64_t)B * H, n_train, d, (flags & FP8ATTN_INPUT_FP16) != 0, key_dest, k_fp8,
+                              n_train * (int64_t)d, stream);
         if (rc != FP8ATTN_OK) return rc;
     }
     return launch_quantize_qkv(q_train, k, v, q_test, (int64_t)B * H, n_train * (int64_t)d,

@@ -58,8 +58,9 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
 
 // key_order.cu
 // dest[b,h,r] = the row that key r of head (b,h) moves to: the keys of largest norm first.
+// norm_scratch: device memory for one fp32 per key, the heads norm_stride_bytes apart.
 int launch_key_order(const void* k16, int64_t n_heads, int64_t n_train, int d, bool half, int32_t* dest,
-                     cudaStream_t stream);
+                     void* norm_scratch, int64_t norm_stride_bytes, cudaStream_t stream);
 // out[b,h,dest[b,h,r],:] = x[b,h,r,:] for a 16-bit tensor
 int launch_reorder_rows(const void* x16, int64_t n_heads, int64_t rows, int d, const int32_t* dest, void* out16,
                         cudaStream_t stream);

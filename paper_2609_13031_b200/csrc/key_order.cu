@@ -50,9 +50,10 @@ __device__ __forceinline__ float sumsq8(uint4 v) {
 }
 
 // One 16-byte vector per thread, kD / 8 neighbouring threads per row.  grid: (blocks, heads).
+// `norm`: rows fp32 bit patterns per head, heads norm_stride words apart.
 template <bool kHalf, int kD>
 __global__ void __launch_bounds__(256) key_norm_kernel(const uint4* __restrict__ k, int64_t rows,
-                                                      uint32_t* __restrict__ dest) {
+                                                      uint32_t* __restrict__ norm, int64_t norm_stride) {
     constexpr int kVecs = kD / 8;
     const int64_t vec = (int64_t)blockIdx.x * 256 + threadIdx.x;
     const int64_t row = vec / kVecs;
@@ -60,24 +61,30 @@ __global__ void __launch_bounds__(256) key_norm_kernel(const uint4* __restrict__
     if (row < rows) s = sumsq8<kHalf>(k[(int64_t)blockIdx.y * rows * kVecs + vec]);
 #pragma unroll
     for (int o = kVecs / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (row < rows && vec % kVecs == 0) dest[(int64_t)blockIdx.y * rows + row] = __float_as_uint(s);
+    if (row < rows && vec % kVecs == 0) norm[(int64_t)blockIdx.y * norm_stride + row] = __float_as_uint(s);
 }
 
-// One block per head.  On entry dest holds the rows' norms (fp32 bit patterns, non-negative, so
-// they order like unsigned integers); on exit the destination row of every row.  The rows at or
-// above the threshold bin are collected in a list (at most kMaxFirst: where more rows than that
-// share the leading bins, the norms single out no small group and the order is left alone),
-// the list is sorted, and every row finds its place by a binary search: a listed row goes to
-// its rank in the list, any other row r to r + (listed rows behind it).
+// grid: (kOrderBlocks, heads).  `norm` holds the rows' squared norms (fp32 bit patterns,
+// non-negative, so they order like unsigned integers).  Every block of a head works out the
+// same threshold and the same list, and writes the destinations of its own share of the rows:
+// the rows at or above the threshold bin are collected in a list (at most kMaxFirst: where more
+// rows than that share the leading bins, the norms single out no small group and the order is
+// left alone), the list is sorted, and every row finds its place by a binary search: a listed
+// row goes to its rank in the list, any other row r to r + (listed rows behind it).
 constexpr int kMaxFirst = 2048;
 constexpr int kSample = 8;
+constexpr int kOrderBlocks = 16;
 
-__global__ void __launch_bounds__(kOrderThreads) key_order_kernel(int64_t rows, uint32_t* __restrict__ dest) {
+__global__ void __launch_bounds__(kOrderThreads)
+key_order_kernel(int64_t rows, const uint32_t* __restrict__ norm, int64_t norm_stride, uint32_t* __restrict__ dest) {
     __shared__ uint32_t hist[kBins];
     __shared__ uint32_t suffix[kOrderThreads];
     __shared__ uint32_t list[kMaxFirst];
     __shared__ uint32_t threshold_bin, first_count;
-    uint32_t* d = dest + (int64_t)blockIdx.x * rows;
+    const uint32_t* d = norm + (int64_t)blockIdx.y * norm_stride;
+    uint32_t* out = dest + (int64_t)blockIdx.y * rows;
+    // this block's share of the rows
+    const int64_t r0 = rows * blockIdx.x / kOrderBlocks, r1 = rows * (blockIdx.x + 1) / kOrderBlocks;
     const int tid = threadIdx.x;
     for (int i = tid; i < kBins; i += kOrderThreads) hist[i] = 0u;
     if (tid == 0) first_count = 0u;
@@ -133,7 +140,7 @@ __global__ void __launch_bounds__(kOrderThreads) key_order_kernel(int64_t rows, 
     __syncthreads();
     const uint32_t count = first_count;
     if (count > (uint32_t)kMaxFirst || count == (uint32_t)rows) {
-        for (int64_t i = tid; i < rows; i += kOrderThreads) d[i] = (uint32_t)i;
+        for (int64_t i = r0 + tid; i < r1; i += kOrderThreads) out[i] = (uint32_t)i;
         return;
     }
     // bitonic sort of the list, padded with the largest value
@@ -152,7 +159,7 @@ __global__ void __launch_bounds__(kOrderThreads) key_order_kernel(int64_t rows, 
             __syncthreads();
         }
     }
-    for (int64_t i = tid; i < rows; i += kOrderThreads) {
+    for (int64_t i = r0 + tid; i < r1; i += kOrderThreads) {
         // listed rows below i (lower bound of i in the sorted list)
         int lo = 0, hi = (int)count;
         while (lo < hi) {
@@ -160,7 +167,7 @@ __global__ void __launch_bounds__(kOrderThreads) key_order_kernel(int64_t rows, 
             if (list[mid] < (uint32_t)i) lo = mid + 1; else hi = mid;
         }
         const bool listed = lo < (int)count && list[lo] == (uint32_t)i;
-        d[i] = listed ? (uint32_t)lo : (uint32_t)i + (count - (uint32_t)lo);
+        out[i] = listed ? (uint32_t)lo : (uint32_t)i + (count - (uint32_t)lo);
     }
 }
 
@@ -179,22 +186,24 @@ __global__ void __launch_bounds__(256) reorder_rows_kernel(const uint4* __restri
 }  // namespace
 
 int launch_key_order(const void* k16, int64_t n_heads, int64_t n_train, int d, bool half, int32_t* dest,
-                     cudaStream_t stream) {
+                     void* norm_scratch, int64_t norm_stride_bytes, cudaStream_t stream) {
     if (n_heads <= 0 || n_train <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     const int64_t vecs = n_train * (d / 8);
     const dim3 grid((unsigned)((vecs + 255) / 256), (unsigned)n_heads);
     const uint4* k = static_cast<const uint4*>(k16);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(dest);
+    uint32_t* norm = static_cast<uint32_t*>(norm_scratch);
+    const int64_t stride = norm_stride_bytes / 4;
     if (d == 64) {
-        if (half) key_norm_kernel<true, 64><<<grid, 256, 0, stream>>>(k, n_train, dst);
-        else key_norm_kernel<false, 64><<<grid, 256, 0, stream>>>(k, n_train, dst);
+        if (half) key_norm_kernel<true, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+        else key_norm_kernel<false, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
     } else {
-        if (half) key_norm_kernel<true, 128><<<grid, 256, 0, stream>>>(k, n_train, dst);
-        else key_norm_kernel<false, 128><<<grid, 256, 0, stream>>>(k, n_train, dst);
+        if (half) key_norm_kernel<true, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+        else key_norm_kernel<false, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
     }
     count_launch();
-    key_order_kernel<<<(unsigned)n_heads, kOrderThreads, 0, stream>>>(n_train, dst);
+    key_order_kernel<<<dim3(kOrderBlocks, (unsigned)n_heads), kOrderThreads, 0, stream>>>(
+        n_train, norm, stride, reinterpret_cast<uint32_t*>(dest));
     count_launch();
     return cudaGetLastError() == cudaSuccess ? FP8ATTN_OK : FP8ATTN_ERR_CUDA;
 }
