@@ -522,6 +522,9 @@ def main():
         peak_fp8 = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops_sustained"]
         peak_fp8_burst = NOMINAL_FP8_OVER_BF16 * peaks["bf16_tflops"]
         quant_bytes = w.B * w.H * w.d * (5 * 3 * w.n_train + 3 * w.n_test)
+        if order_keys:
+            # one more pass over K for the row norms, the norms written and read, the row map written and read twice
+            quant_bytes += w.B * w.H * w.n_train * (2 * w.d + 4 * 5)
         # secondary roofline: the exponential path.  One exponential per score; the MUFU
         # evaluates 16 per clock per SM, and with the kernel's share of them on the FMA pipe
         # the limit is 16 / (1 - share).  Clock = the median SM clock sampled during the timed steps.
