@@ -137,9 +137,11 @@ int fp8attn_quantize_qkv_ex(const void* q_train, const void* k, const void* v, c
  *   key_dest  out int32 [B,H,n_train] (device): the row that key r of head (b,h) was moved to,
  *             a permutation per head.  K8 and V8 are written in that order
  *             (k_fp8[b,h,key_dest[b,h,r],:] = code of k[b,h,r,:]); scales, Q8 and Q_test8 are
- *             those of fp8attn_quantize_qkv_ex.  It takes the two-launch form plus two small
- *             launches for the order (which stage the key norms in the k_fp8 buffer before the
- *             codes are written there).  Other arguments and flags as fp8attn_quantize_qkv_ex.
+ *             those of fp8attn_quantize_qkv_ex.  It takes the two-launch form (whose maximum
+ *             pass also leaves the key norms in the k_fp8 buffer, until the codes are written
+ *             there) with one small launch for the order in between; with FP8ATTN_SCALES_GIVEN
+ *             a pass of its own computes the norms.  Other arguments and flags as
+ *             fp8attn_quantize_qkv_ex.
  *
  * The forward calls need nothing: pass the reordered K8 and V8.  Measured on B200: 3.5 % of
  * the attention time on tables whose row norms vary (log-normal, sigma 0.5), nothing on

@@ -152,13 +152,6 @@ int quantize_qkv_impl(const void* q_train, const void* k, const void* v, const v
     uint32_t* amax = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsAmaxOffset);
     char* ws = static_cast<char*>(workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (key_dest != nullptr) {
-        // the key norms go through the K8 buffer (d bytes per key, of which four are used),
-        // which the conversion overwrites afterwards
-        rc = launch_key_order(k, (int64_t)B * H, n_train, d, (flags & FP8ATTN_INPUT_FP16) != 0, key_dest, k_fp8,
-                              n_train * (int64_t)d, stream);
-        if (rc != FP8ATTN_OK) return rc;
-    }
     return launch_quantize_qkv(q_train, k, v, q_test, (int64_t)B * H, n_train * (int64_t)d,
                                n_test * (int64_t)d, q_train_fp8, k_fp8, v_fp8, q_test_fp8, scale_q, scale_k,
                                scale_v, amax, flags, reinterpret_cast<uint32_t*>(ws + kWsStatusOffset),

@@ -54,13 +54,14 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
                         float* scale_v, uint32_t* amax_bits, uint32_t flags, uint32_t* status,
                         uint32_t* counters, float* partial, cudaStream_t stream,
-                        const int32_t* key_dest = nullptr, int d = 64);
+                        int32_t* key_dest = nullptr, int d = 64);
 
 // key_order.cu
 // dest[b,h,r] = the row that key r of head (b,h) moves to: the keys of largest norm first.
-// norm_scratch: device memory for one fp32 per key, the heads norm_stride_bytes apart.
+// norm_scratch: device memory for one fp32 per key (its squared norm), the heads
+// norm_stride_bytes apart; compute_norms: fill it from k16 first (else it is filled already).
 int launch_key_order(const void* k16, int64_t n_heads, int64_t n_train, int d, bool half, int32_t* dest,
-                     void* norm_scratch, int64_t norm_stride_bytes, cudaStream_t stream);
+                     void* norm_scratch, int64_t norm_stride_bytes, bool compute_norms, cudaStream_t stream);
 // out[b,h,dest[b,h,r],:] = x[b,h,r,:] for a 16-bit tensor
 int launch_reorder_rows(const void* x16, int64_t n_heads, int64_t rows, int d, const int32_t* dest, void* out16,
                         cudaStream_t stream);

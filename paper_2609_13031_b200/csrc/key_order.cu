@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(256) reorder_rows_kernel(const uint4* __restri
 }  // namespace
 
 int launch_key_order(const void* k16, int64_t n_heads, int64_t n_train, int d, bool half, int32_t* dest,
-                     void* norm_scratch, int64_t norm_stride_bytes, cudaStream_t stream) {
+                     void* norm_scratch, int64_t norm_stride_bytes, bool compute_norms, cudaStream_t stream) {
     if (n_heads <= 0 || n_train <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     const int64_t vecs = n_train * (d / 8);
@@ -194,14 +194,16 @@ int launch_key_order(const void* k16, int64_t n_heads, int64_t n_train, int d, b
     const uint4* k = static_cast<const uint4*>(k16);
     uint32_t* norm = static_cast<uint32_t*>(norm_scratch);
     const int64_t stride = norm_stride_bytes / 4;
-    if (d == 64) {
-        if (half) key_norm_kernel<true, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
-        else key_norm_kernel<false, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
-    } else {
-        if (half) key_norm_kernel<true, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
-        else key_norm_kernel<false, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+    if (compute_norms) {
+        if (d == 64) {
+            if (half) key_norm_kernel<true, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+            else key_norm_kernel<false, 64><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+        } else {
+            if (half) key_norm_kernel<true, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+            else key_norm_kernel<false, 128><<<grid, 256, 0, stream>>>(k, n_train, norm, stride);
+        }
+        count_launch();
     }
-    count_launch();
     key_order_kernel<<<dim3(kOrderBlocks, (unsigned)n_heads), kOrderThreads, 0, stream>>>(
         n_train, norm, stride, reinterpret_cast<uint32_t*>(dest));
     count_launch();

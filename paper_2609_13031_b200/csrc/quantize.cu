@@ -62,12 +62,30 @@ template <> struct In16<true> {
 
 // One block's share of max |x| over head blockIdx.y (vecs_per_head 16-byte vectors),
 // merged into amax_bits[blockIdx.y].
-template <bool kHalf>
+// With kNorm it also leaves the squared norm of every row (vecs_per_row 16-byte vectors, 8 or
+// 16; fp32 bit pattern) in row_norm[row] of the head: the vectors of a row sit in neighbouring
+// lanes, whose loop conditions agree (all bounds are multiples of the row length), so the lanes
+// of a row add up under a mask of their own.
+template <bool kHalf, bool kNorm = false>
 __device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t vecs_per_head,
-                                            uint32_t* __restrict__ amax_bits) {
+                                            uint32_t* __restrict__ amax_bits,
+                                            uint32_t* __restrict__ row_norm = nullptr, int vecs_per_row = 8) {
     using T = In16<kHalf>;
     using V2 = typename T::V2;
     auto am = [](uint32_t a, uint32_t b) { return __hmax2(__habs2(T::as2(a)), __habs2(T::as2(b))); };
+    const uint32_t row_mask = (vecs_per_row == 16 ? 0xffffu : 0xffu) << (threadIdx.x & 31 & ~(vecs_per_row - 1));
+    auto norm_of = [&](const uint4& v, int64_t vec) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float q = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = T::lo(w[k]), hi = T::hi(w[k]);
+            q = fmaf(lo, lo, q);
+            q = fmaf(hi, hi, q);
+        }
+        for (int o = vecs_per_row >> 1; o > 0; o >>= 1) q += __shfl_xor_sync(row_mask, q, o);
+        if ((vec & (vecs_per_row - 1)) == 0) row_norm[vec / vecs_per_row] = __float_as_uint(q);
+    };
     const uint4* xh = x + (int64_t)blockIdx.y * vecs_per_head;
     V2 m = T::as2(0u);
     int64_t stride = (int64_t)gridDim.x * kThreads;
@@ -75,6 +93,12 @@ __device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t
     for (; i + 3 * stride < vecs_per_head; i += 4 * stride) {
         uint4 a = ld_nc_v4(xh + i), b = ld_nc_v4(xh + i + stride);
         uint4 c = ld_nc_v4(xh + i + 2 * stride), e = ld_nc_v4(xh + i + 3 * stride);
+        if (kNorm) {
+            norm_of(a, i);
+            norm_of(b, i + stride);
+            norm_of(c, i + 2 * stride);
+            norm_of(e, i + 3 * stride);
+        }
         V2 m0 = am(a.x, a.y), m1 = am(a.z, a.w), m2 = am(b.x, b.y), m3 = am(b.z, b.w);
         V2 m4 = am(c.x, c.y), m5 = am(c.z, c.w), m6 = am(e.x, e.y), m7 = am(e.z, e.w);
         m = __hmax2(m, __hmax2(__hmax2(__hmax2(m0, m1), __hmax2(m2, m3)),
@@ -82,6 +106,7 @@ __device__ __forceinline__ void absmax_body(const uint4* __restrict__ x, int64_t
     }
     for (; i < vecs_per_head; i += stride) {
         uint4 a = ld_nc_v4(xh + i);
+        if (kNorm) norm_of(a, i);
         m = __hmax2(m, __hmax2(am(a.x, a.y), am(a.z, a.w)));
     }
     // |x| as a non-negative fp32 bit pattern orders like an unsigned integer
@@ -219,10 +244,17 @@ struct QuantBatch {
     int pairs_per_row_shift;      // log2(d / 16)
 };
 
-template <bool kHalf>
-__global__ void __launch_bounds__(kThreads) absmax_batch_kernel(const QuantBatch b) {
+// kNorm: the pass over K (z = 1) also leaves the keys' squared norms in key_norm (one word per
+// key, the heads key_norm_stride words apart).
+template <bool kHalf, bool kNorm = false>
+__global__ void __launch_bounds__(kThreads)
+absmax_batch_kernel(const QuantBatch b, uint32_t* key_norm = nullptr, int64_t key_norm_stride = 0) {
     const int z = blockIdx.z;
-    if (b.amax_acc[z] != nullptr && b.pairs_per_head[z] > 0)
+    if (b.amax_acc[z] == nullptr || b.pairs_per_head[z] <= 0) return;
+    if (kNorm && z == 1)
+        absmax_body<kHalf, true>(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z],
+                                 key_norm + (int64_t)blockIdx.y * key_norm_stride, 2 << b.pairs_per_row_shift);
+    else
         absmax_body<kHalf>(b.x[z], b.pairs_per_head[z] * 2, b.amax_acc[z]);
 }
 
@@ -427,8 +459,7 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
                         int64_t n_heads, int64_t elems_train, int64_t elems_test, void* q_train_fp8,
                         void* k_fp8, void* v_fp8, void* q_test_fp8, float* scale_q, float* scale_k,
                         float* scale_v, uint32_t* amax_bits, uint32_t flags, uint32_t* status,
-                        uint32_t* counters, float* partial, cudaStream_t stream, const int32_t* key_dest,
-                        int d) {
+                        uint32_t* counters, float* partial, cudaStream_t stream, int32_t* key_dest, int d) {
     if (n_heads <= 0) return FP8ATTN_OK;
     if (n_heads > 65535) return FP8ATTN_ERR_UNSUPPORTED;
     QuantBatch b;
@@ -490,10 +521,27 @@ int launch_quantize_qkv(const void* q_train, const void* k, const void* v, const
     if (!(flags & FP8ATTN_SCALES_GIVEN) &&
         cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 3 * n_heads, stream) != cudaSuccess)
         return FP8ATTN_ERR_CUDA;
+    // A key order is built between the two passes: the keys' norms come out of the maximum pass
+    // (or, where the scales are given and there is none, out of a pass of their own) and sit in
+    // the K8 buffer until the conversion overwrites them.
+    uint32_t* key_norm = reinterpret_cast<uint32_t*>(k_fp8);
+    const int64_t key_norm_stride = elems_train / 4;        // K8 bytes per head, in words
+    const int64_t keys = elems_train / d;
     if (elems_train > 0 && !(flags & FP8ATTN_SCALES_GIVEN)) {
-        if (half) absmax_batch_kernel<true><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
-        else absmax_batch_kernel<false><<<dim3(bx, (unsigned)n_heads, 4), kThreads, 0, stream>>>(b);
+        const dim3 grid(bx, (unsigned)n_heads, 4);
+        if (key_dest != nullptr) {
+            if (half) absmax_batch_kernel<true, true><<<grid, kThreads, 0, stream>>>(b, key_norm, key_norm_stride);
+            else absmax_batch_kernel<false, true><<<grid, kThreads, 0, stream>>>(b, key_norm, key_norm_stride);
+        } else {
+            if (half) absmax_batch_kernel<true><<<grid, kThreads, 0, stream>>>(b);
+            else absmax_batch_kernel<false><<<grid, kThreads, 0, stream>>>(b);
+        }
         count_launch();
+    }
+    if (key_dest != nullptr && elems_train > 0) {
+        const int rc = launch_key_order(k, n_heads, keys, d, half, key_dest, key_norm,
+                                        key_norm_stride * 4, (flags & FP8ATTN_SCALES_GIVEN) != 0, stream);
+        if (rc != FP8ATTN_OK) return rc;
     }
     if (half) quantize_batch_kernel<true><<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
     else quantize_batch_kernel<false><<<dim3(bx, (unsigned)n_heads, tensors), kThreads, 0, stream>>>(b);
